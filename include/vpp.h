@@ -1,0 +1,168 @@
+/*
+ * vpp.h -- C ABI of the B200 chunked-prefill attention library.
+ *
+ * The operation is the attention step inside a chunked prefill (the paper's
+ * Eq. 1 with the causal rule of its Transformer background section, applied
+ * per chunk as described in its "Chunked Prefill Pipeline Parallelism"
+ * section): a packed chunk of query rows attends causally to itself and to
+ * the whole prefix already held in a (paged) KV cache.  For request r with
+ * prefix_len P and chunk_len C, query row i (0 <= i < C) of q-head h sits at
+ * absolute position p = P + i and sees cached keys 0..p (inclusive) of
+ * kv-head h / (num_q_heads / num_kv_heads):
+ *
+ *     s_j = softmax_scale * <q, k_j>,  out = sum_j softmax(s)_j * v_j,
+ *     lse = ln sum_j exp(s_j)
+ *
+ * The cost of one chunk grows linearly with its prefix length: this is the
+ * per-chunk imbalance the paper's V-shaped virtual-stage layout is built
+ * around (its Eq. 2-3).
+ *
+ * General rules
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".
+ *  - The caller owns every buffer; the library allocates no device memory
+ *    in the entry points declared here.
+ *  - All work is enqueued on `stream`; no entry point synchronises.
+ *  - Entry points return VPP_OK or a negative vpp_status; vpp_last_error()
+ *    gives a thread-local message for the most recent failure.
+ *  - There is no CPU fallback: unsupported shapes return VPP_ERR_UNSUPPORTED.
+ */
+#ifndef VPP_H_
+#define VPP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    VPP_OK = 0,
+    VPP_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad stride or alignment */
+    VPP_ERR_UNSUPPORTED = -2, /* head dims / block size this build has no kernel for   */
+    VPP_ERR_WORKSPACE = -3,   /* workspace missing or smaller than the size query      */
+    VPP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                   */
+    VPP_ERR_TIMEOUT = -5      /* (device status only) a bounded device wait expired    */
+} vpp_status;
+
+/* Values the device writes to *status (0 = success). */
+enum {
+    VPP_DEV_OK = 0,
+    VPP_DEV_BAD_LENGTHS = 1,  /* prefix_len/chunk_len negative, beyond max_seq_len, or sum != total_q */
+    VPP_DEV_BAD_BLOCK = 2,    /* a block_table entry that is needed lies outside [0, num_blocks)       */
+    VPP_DEV_TIMEOUT = 3       /* a bounded wait inside a kernel expired; outputs are undefined         */
+};
+
+typedef void *vpp_stream_t; /* a cudaStream_t */
+
+/*
+ * Arguments of vpp_chunk_attn_fwd.
+ *
+ * q            bf16 [total_q, num_q_heads, head_dim_qk], dense, packed request-major: the rows of
+ *              request r start at sum_{r' < r} chunk_len[r'].  16-byte aligned.
+ * k_cache      bf16; element (block b, slot t, kv-head g, feature d) lives at
+ *              b*k_block_stride + t*k_token_stride + g*k_head_stride + d   (strides in ELEMENTS,
+ *              feature stride 1; each stride a multiple of 8 elements; base 16-byte aligned).
+ *              The usual layout [num_blocks, block_size, Hkv, Dqk] has strides
+ *              (block_size*Hkv*Dqk, Hkv*Dqk, Dqk).
+ * v_cache      same addressing with the v_* strides and head_dim_v features.  It may alias k_cache
+ *              (absorbed MLA: V is the first head_dim_v features of each K row).
+ *              The cache must ALREADY hold positions [0, prefix_len+chunk_len) of every request:
+ *              the chunk's own K/V are written before this call.  Slots past that point inside a
+ *              request's last block may hold anything (NaN included) and blocks the block table
+ *              does not name are never read.
+ * block_table  int32 [num_reqs, max_blocks_per_req]: physical block of logical block j of request r.
+ *              NULL means contiguous: request r is "block" r and block_size is ignored (slot = token).
+ * prefix_len   int32 [num_reqs], tokens of the request already cached before this chunk.
+ * chunk_len    int32 [num_reqs], query rows of the request in this call (0 allowed).
+ * total_q      host copy of sum(chunk_len); sizes out, lse and the workspace.
+ * max_seq_len  host upper bound on prefix_len[r] + chunk_len[r].
+ * num_kv_splits  0: the library decides; 1: never split the key range; S > 1: split the key range of
+ *              every query tile into up to S parts and merge them (split-KV).
+ * out          bf16 [total_q, num_q_heads, head_dim_v], 16-byte aligned.
+ * lse          fp32 [total_q, num_q_heads], natural log of sum_j exp(softmax_scale * <q,k_j>) over
+ *              the visible keys; may be NULL.
+ * workspace    at least vpp_chunk_attn_workspace_size(args) bytes, 256-byte aligned.  Contents need
+ *              no initialisation and are clobbered.  Two calls that overlap on the GPU need two
+ *              workspaces.
+ * status       optional device int32.  Zeroed by the call; a nonzero VPP_DEV_* value afterwards
+ *              means a device-side check failed and out/lse must not be used.
+ *
+ * Supported shapes: (head_dim_qk, head_dim_v) = (128, 128) with num_q_heads % num_kv_heads == 0, and
+ * (576, 512) with num_kv_heads == 1; block_size a power of two >= 16 (or block_table == NULL).
+ */
+typedef struct {
+    const void *q;
+    const void *k_cache;
+    const void *v_cache;
+    int64_t k_block_stride, k_token_stride, k_head_stride;
+    int64_t v_block_stride, v_token_stride, v_head_stride;
+    const int32_t *block_table;
+    const int32_t *prefix_len;
+    const int32_t *chunk_len;
+    int32_t num_reqs;
+    int32_t max_blocks_per_req;
+    int32_t block_size;
+    int32_t num_blocks;
+    int32_t total_q;
+    int32_t max_seq_len;
+    int32_t num_q_heads;
+    int32_t num_kv_heads;
+    int32_t head_dim_qk;
+    int32_t head_dim_v;
+    float softmax_scale;
+    int32_t num_kv_splits;
+    void *out;
+    float *lse;
+    void *workspace;
+    size_t workspace_bytes;
+    int32_t *status;
+} vpp_chunk_attn_args;
+
+/*
+ * Bytes of workspace vpp_chunk_attn_fwd needs for these arguments (only the host-side scalar
+ * fields are read).  Pure host arithmetic apart from one cached device-attribute query.
+ * Returns 0 if the arguments are invalid.
+ */
+size_t vpp_chunk_attn_workspace_size(const vpp_chunk_attn_args *args);
+
+/*
+ * Chunked-prefill attention forward (the operation defined at the top of this file).
+ * Enqueues: a work-decomposition kernel (query tiles x heads x key-range splits, ordered by
+ * decreasing cost), the persistent attention kernel, and, when the key range was split, the
+ * merge kernel.  Returns after enqueueing.
+ * Errors: VPP_ERR_INVALID_ARG / VPP_ERR_UNSUPPORTED / VPP_ERR_WORKSPACE before anything is
+ * enqueued; VPP_ERR_CUDA if a launch fails.
+ */
+vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args *args, vpp_stream_t stream);
+
+/*
+ * Merge of partial attention results computed over disjoint key sets (split-KV, or the
+ * per-device partials of a context-parallel prefix):
+ *     lse = ln sum_s exp(lse_s),   out = sum_s exp(lse_s - lse) * o_s
+ * where each o_s is already normalised by its own split.  A split with lse_s = -inf contributes
+ * nothing; a row whose splits are all -inf gets out = 0, lse = -inf.
+ *
+ * o_parts    fp32 [num_splits, total_q, num_q_heads, head_dim_v]
+ * lse_parts  fp32 [num_splits, total_q, num_q_heads]
+ * out        bf16 [total_q, num_q_heads, head_dim_v]
+ * lse        fp32 [total_q, num_q_heads] or NULL
+ * head_dim_v must be a multiple of 8; pointers 16-byte aligned.
+ */
+vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t num_splits,
+                         int32_t total_q, int32_t num_q_heads, int32_t head_dim_v, void *out,
+                         float *lse, vpp_stream_t stream);
+
+/* Static description of a status code. */
+const char *vpp_status_string(vpp_status s);
+
+/* Thread-local detail of the last failure on this host thread ("" if none). */
+const char *vpp_last_error(void);
+
+/* Number of kernels the last successful vpp_chunk_attn_fwd on this host thread enqueued. */
+int32_t vpp_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VPP_H_ */

@@ -1,0 +1,160 @@
+"""ctypes binding of the C ABI in include/vpp.h (argument marshalling only).
+
+Every step of the attention path runs in the CUDA library; PyTorch is used for device memory and
+streams.  There is no CPU fallback: if the shared library is missing or cannot be loaded, calls raise.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvpp_chunk_attn.so")
+
+VPP_OK = 0
+VPP_ERR_INVALID_ARG = -1
+VPP_ERR_UNSUPPORTED = -2
+VPP_ERR_WORKSPACE = -3
+VPP_ERR_CUDA = -4
+VPP_ERR_TIMEOUT = -5
+
+EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_status_string",
+           "vpp_last_error", "vpp_last_launch_count"]
+
+
+class VppError(RuntimeError):
+    def __init__(self, status, detail):
+        super().__init__("vpp status %d: %s" % (status, detail))
+        self.status = status
+
+
+class ChunkAttnArgs(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+        ("k_block_stride", ctypes.c_int64), ("k_token_stride", ctypes.c_int64), ("k_head_stride", ctypes.c_int64),
+        ("v_block_stride", ctypes.c_int64), ("v_token_stride", ctypes.c_int64), ("v_head_stride", ctypes.c_int64),
+        ("block_table", ctypes.c_void_p), ("prefix_len", ctypes.c_void_p), ("chunk_len", ctypes.c_void_p),
+        ("num_reqs", ctypes.c_int32), ("max_blocks_per_req", ctypes.c_int32), ("block_size", ctypes.c_int32),
+        ("num_blocks", ctypes.c_int32), ("total_q", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
+        ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim_qk", ctypes.c_int32),
+        ("head_dim_v", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("num_kv_splits", ctypes.c_int32),
+        ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library():
+    """Load libvpp_chunk_attn.so (raises if it has not been built: there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: run `python -m paper_2608_26523_b200.build`" % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.vpp_chunk_attn_workspace_size.restype = ctypes.c_size_t
+        lib.vpp_chunk_attn_workspace_size.argtypes = [ctypes.POINTER(ChunkAttnArgs)]
+        lib.vpp_chunk_attn_fwd.restype = ctypes.c_int
+        lib.vpp_chunk_attn_fwd.argtypes = [ctypes.POINTER(ChunkAttnArgs), ctypes.c_void_p]
+        lib.vpp_lse_merge.restype = ctypes.c_int
+        lib.vpp_lse_merge.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_void_p]
+        lib.vpp_status_string.restype = ctypes.c_char_p
+        lib.vpp_status_string.argtypes = [ctypes.c_int]
+        lib.vpp_last_error.restype = ctypes.c_char_p
+        lib.vpp_last_launch_count.restype = ctypes.c_int32
+        _lib = lib
+    return _lib
+
+
+def _check(rc):
+    if rc != VPP_OK:
+        lib = load_library()
+        raise VppError(rc, "%s: %s" % (lib.vpp_status_string(rc).decode(), lib.vpp_last_error().decode()))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def make_args(q, k_cache, v_cache, block_table, prefix_len, chunk_len, block_size, max_seq_len,
+              softmax_scale, num_kv_splits=0, out=None, lse=None, workspace=None, status=None,
+              total_q=None, head_dim_v=None):
+    """Fill a vpp_chunk_attn_args from tensors.
+
+    q [T, Hq, Dqk] bf16; k_cache/v_cache [num_blocks, block_size, Hkv, D] bf16 (any strides with a
+    contiguous last dim; v may be a view of k); block_table int32 [R, max_blocks] or None.
+    """
+    a = ChunkAttnArgs()
+    a.q, a.k_cache, a.v_cache = _ptr(q), _ptr(k_cache), _ptr(v_cache)
+    ks, vs = k_cache.stride(), v_cache.stride()
+    assert ks[3] == 1 and vs[3] == 1 and q.is_contiguous()
+    a.k_block_stride, a.k_token_stride, a.k_head_stride = ks[0], ks[1], ks[2]
+    a.v_block_stride, a.v_token_stride, a.v_head_stride = vs[0], vs[1], vs[2]
+    a.block_table = _ptr(block_table)
+    a.prefix_len, a.chunk_len = _ptr(prefix_len), _ptr(chunk_len)
+    a.num_reqs = prefix_len.numel()
+    a.max_blocks_per_req = 0 if block_table is None else block_table.shape[1]
+    a.block_size = int(block_size)
+    a.num_blocks = k_cache.shape[0]
+    a.total_q = q.shape[0] if total_q is None else int(total_q)
+    a.max_seq_len = int(max_seq_len)
+    a.num_q_heads, a.num_kv_heads = q.shape[1], k_cache.shape[2]
+    a.head_dim_qk = q.shape[2]
+    a.head_dim_v = v_cache.shape[3] if head_dim_v is None else int(head_dim_v)
+    a.softmax_scale = float(softmax_scale)
+    a.num_kv_splits = int(num_kv_splits)
+    a.out, a.lse = _ptr(out), _ptr(lse)
+    a.workspace = _ptr(workspace)
+    a.workspace_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    a.status = _ptr(status)
+    return a
+
+
+def vpp_chunk_attn_workspace_size(args):
+    return int(load_library().vpp_chunk_attn_workspace_size(ctypes.byref(args)))
+
+
+def vpp_chunk_attn_fwd(args, stream=None):
+    """Enqueue chunked-prefill attention on `stream` (default: torch's current stream)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_chunk_attn_fwd(ctypes.byref(args), ctypes.c_void_p(stream)))
+
+
+def vpp_lse_merge(o_parts, lse_parts, out, lse=None, stream=None):
+    """out/lse <- merge of o_parts [S,T,Hq,Dv] fp32 and lse_parts [S,T,Hq] fp32."""
+    S, T, Hq, Dv = o_parts.shape
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_lse_merge(_ptr(o_parts), _ptr(lse_parts), S, T, Hq, Dv, _ptr(out), _ptr(lse),
+                                        ctypes.c_void_p(stream)))
+
+
+def vpp_last_launch_count():
+    return int(load_library().vpp_last_launch_count())
+
+
+class ChunkAttn:
+    """Convenience wrapper that owns out / lse / workspace / status for one Problem-shaped launch."""
+
+    def __init__(self, prob, num_kv_splits=0, want_lse=True):
+        dev = prob.q.device
+        self.prob = prob
+        self.out = torch.empty((prob.total_q, prob.num_q_heads, prob.head_dim_v), dtype=torch.bfloat16, device=dev)
+        self.lse = torch.empty((prob.total_q, prob.num_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.args = make_args(prob.q, prob.k_cache, prob.v_cache, prob.block_table, prob.prefix_len,
+                              prob.chunk_len, prob.block_size, prob.max_seq_len, prob.scale,
+                              num_kv_splits=num_kv_splits, out=self.out, lse=self.lse, status=self.status,
+                              head_dim_v=prob.head_dim_v)
+        n = vpp_chunk_attn_workspace_size(self.args)
+        self.workspace = torch.empty(max(n, 256), dtype=torch.uint8, device=dev)
+        self.args.workspace = _ptr(self.workspace)
+        self.args.workspace_bytes = self.workspace.numel()
+
+    def run(self, stream=None):
+        vpp_chunk_attn_fwd(self.args, stream)
+        return self.out, self.lse

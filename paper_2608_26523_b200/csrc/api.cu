@@ -1,0 +1,371 @@
+// Host side of the C ABI declared in include/vpp.h: argument validation, workspace layout,
+// tensor-map construction and kernel launches.  Nothing here synchronises or allocates device memory.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "../../include/vpp.h"
+#include "attn_simple.cuh"
+#include "common.cuh"
+#include "merge.cuh"
+#include "prep.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+thread_local int32_t g_launches = 0;
+
+vpp_status fail(vpp_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- device facts, cached per device -------------------------------------------------------------
+struct DeviceInfo {
+    bool ready = false;
+    int sm_count = 0;
+    bool attrs_set = false;
+};
+std::mutex g_mu;
+DeviceInfo g_dev[64];
+
+int sm_count_or_default() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return 148;
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g_dev[dev].ready) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            n = 148;
+        }
+        g_dev[dev].sm_count = n;
+        g_dev[dev].ready = true;
+    }
+    return g_dev[dev].sm_count;
+}
+
+// ---- tensor maps ------------------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                              CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+    static EncodeFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+// bf16 tensor, innermost dimension contiguous, 128-byte swizzle, zero fill out of bounds.
+bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+               const uint32_t* box) {
+    EncodeFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t gd[5], gs[4];
+    cuuint32_t bx[5], es[5];
+    for (int i = 0; i < rank; ++i) {
+        gd[i] = dims[i];
+        bx[i] = box[i];
+        es[i] = 1;
+        if (i > 0) gs[i - 1] = strides_bytes[i - 1];
+    }
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gd, gs, bx, es,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// ---- validation -------------------------------------------------------------------------------------
+bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+int ilog2(int x) {
+    int s = 0;
+    while ((1 << s) < x) ++s;
+    return s;
+}
+
+enum class Family { kGqa128, kMla576, kNone };
+
+vpp_status validate(const vpp_chunk_attn_args* a, Family* fam) {
+    if (!a) return fail(VPP_ERR_INVALID_ARG, "args is null");
+    if (a->num_reqs < 0 || a->total_q < 0 || a->max_seq_len < 0)
+        return fail(VPP_ERR_INVALID_ARG, "num_reqs, total_q and max_seq_len must be >= 0");
+    if (a->num_q_heads <= 0 || a->num_kv_heads <= 0 || a->num_q_heads % a->num_kv_heads != 0)
+        return fail(VPP_ERR_INVALID_ARG, "num_q_heads (%d) must be a positive multiple of num_kv_heads (%d)",
+                    a->num_q_heads, a->num_kv_heads);
+    if (!(a->softmax_scale > 0.f) || !std::isfinite(a->softmax_scale))
+        return fail(VPP_ERR_INVALID_ARG, "softmax_scale must be positive and finite");
+    if (a->num_kv_splits < 0 || a->num_kv_splits > 64)
+        return fail(VPP_ERR_INVALID_ARG, "num_kv_splits must be in [0, 64]");
+    if (a->head_dim_qk == 128 && a->head_dim_v == 128)
+        *fam = Family::kGqa128;
+    else if (a->head_dim_qk == 576 && a->head_dim_v == 512 && a->num_kv_heads == 1)
+        *fam = Family::kMla576;
+    else
+        return fail(VPP_ERR_UNSUPPORTED, "no kernel for head dims (%d, %d) with %d kv heads", a->head_dim_qk,
+                    a->head_dim_v, a->num_kv_heads);
+    if (a->block_table != nullptr) {
+        if (!is_pow2(a->block_size) || a->block_size < 16)
+            return fail(VPP_ERR_UNSUPPORTED, "block_size %d: need a power of two >= 16", a->block_size);
+        if (a->max_blocks_per_req <= 0 || a->num_blocks <= 0)
+            return fail(VPP_ERR_INVALID_ARG, "paged cache needs max_blocks_per_req > 0 and num_blocks > 0");
+    }
+    return VPP_OK;
+}
+
+vpp_status validate_pointers(const vpp_chunk_attn_args* a) {
+    if (a->num_reqs > 0 && (!a->prefix_len || !a->chunk_len))
+        return fail(VPP_ERR_INVALID_ARG, "prefix_len / chunk_len is null");
+    if (a->total_q > 0 && (!a->q || !a->out || !a->k_cache || !a->v_cache))
+        return fail(VPP_ERR_INVALID_ARG, "q, k_cache, v_cache and out must be non-null");
+    auto mis16 = [](const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+    if (mis16(a->q) || mis16(a->out) || mis16(a->k_cache) || mis16(a->v_cache))
+        return fail(VPP_ERR_INVALID_ARG, "q, out, k_cache and v_cache must be 16-byte aligned");
+    const int64_t st[6] = {a->k_block_stride, a->k_token_stride, a->k_head_stride,
+                           a->v_block_stride, a->v_token_stride, a->v_head_stride};
+    for (int i = 0; i < 6; ++i)
+        if (st[i] <= 0 || st[i] % 8 != 0)
+            return fail(VPP_ERR_INVALID_ARG, "cache strides must be positive multiples of 8 elements");
+    return VPP_OK;
+}
+
+// Upper bound on key-range splits per query tile for this launch.
+int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
+    if (a->num_kv_splits >= 1) return a->num_kv_splits;
+    const long long tiles = (a->total_q + vpp::kTileM - 1) / vpp::kTileM + a->num_reqs;
+    const long long items = tiles * (a->num_q_heads / heads_per_item);
+    const int sms = sm_count_or_default();
+    if (items >= 2ll * sms || items == 0) return 1;
+    long long s = (2ll * sms + items - 1) / items;
+    const long long by_len = (a->max_seq_len / vpp::kTileN) / 4;  // keep at least 4 KV tiles per split
+    if (s > by_len) s = by_len;
+    if (s > 16) s = 16;
+    if (s < 1) s = 1;
+    return static_cast<int>(s);
+}
+
+int heads_per_item(const vpp_chunk_attn_args*, Family) { return 1; }
+
+vpp::WorkspaceLayout layout_for(const vpp_chunk_attn_args* a, Family fam) {
+    vpp::WorkspaceLayout L{};
+    const int S = choose_splits(a, heads_per_item(a, fam));
+    const long long tiles = (a->total_q + vpp::kTileM - 1) / vpp::kTileM + a->num_reqs;
+    L.splits = S;
+    L.max_units = static_cast<int32_t>(tiles * S);
+    size_t off = 0;
+    L.header = off;
+    off = align_up(off + sizeof(vpp::WorkHeader), 256);
+    L.units = off;
+    off = align_up(off + sizeof(vpp::WorkUnit) * static_cast<size_t>(L.max_units > 0 ? L.max_units : 1), 256);
+    L.row_splits = off;  // followed by q_start and tile_start scratch
+    off = align_up(off + sizeof(int32_t) * (static_cast<size_t>(a->total_q) + 2 * (static_cast<size_t>(a->num_reqs) + 1)),
+                   256);
+    L.o_parts = off;
+    if (S > 1)
+        off = align_up(off + sizeof(float) * static_cast<size_t>(S) * a->total_q * a->num_q_heads * a->head_dim_v, 256);
+    L.lse_parts = off;
+    if (S > 1) off = align_up(off + sizeof(float) * static_cast<size_t>(S) * a->total_q * a->num_q_heads, 256);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* vpp_status_string(vpp_status s) {
+    switch (s) {
+        case VPP_OK: return "ok";
+        case VPP_ERR_INVALID_ARG: return "invalid argument";
+        case VPP_ERR_UNSUPPORTED: return "unsupported shape";
+        case VPP_ERR_WORKSPACE: return "workspace missing or too small";
+        case VPP_ERR_CUDA: return "CUDA call failed";
+        case VPP_ERR_TIMEOUT: return "device wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* vpp_last_error(void) { return g_err; }
+int32_t vpp_last_launch_count(void) { return g_launches; }
+
+size_t vpp_chunk_attn_workspace_size(const vpp_chunk_attn_args* a) {
+    Family fam = Family::kNone;
+    if (validate(a, &fam) != VPP_OK) return 0;
+    return layout_for(a, fam).total;
+}
+
+vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    Family fam = Family::kNone;
+    vpp_status st = validate(a, &fam);
+    if (st != VPP_OK) return st;
+    st = validate_pointers(a);
+    if (st != VPP_OK) return st;
+    const vpp::WorkspaceLayout L = layout_for(a, fam);
+    if (!a->workspace || a->workspace_bytes < L.total)
+        return fail(VPP_ERR_WORKSPACE, "workspace: need %zu bytes, got %zu", L.total, a->workspace_bytes);
+    if (reinterpret_cast<uintptr_t>(a->workspace) & 255u)
+        return fail(VPP_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    if (fam == Family::kMla576) return fail(VPP_ERR_UNSUPPORTED, "the (576, 512) kernel is not built yet");
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    g_launches = 0;
+    if (a->status) {
+        if (cudaMemsetAsync(a->status, 0, sizeof(int32_t), stream) != cudaSuccess)
+            return fail(VPP_ERR_CUDA, "memset status: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+    if (a->total_q == 0 || a->num_reqs == 0) return VPP_OK;
+
+    uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+    const bool paged = a->block_table != nullptr;
+    const int B = paged ? a->block_size : a->max_seq_len;
+    const int n_blocks = paged ? a->num_blocks : a->num_reqs;
+    const int box_rows = paged ? (B < vpp::kTileN ? B : vpp::kTileN) : vpp::kTileN;
+
+    // ---- tensor maps ----
+    CUtensorMap tm_q, tm_k, tm_v;
+    {
+        const uint64_t d[3] = {static_cast<uint64_t>(a->head_dim_qk), static_cast<uint64_t>(a->num_q_heads),
+                               static_cast<uint64_t>(a->total_q)};
+        const uint64_t s[2] = {static_cast<uint64_t>(a->head_dim_qk) * 2,
+                               static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2};
+        const uint32_t b[3] = {64, 1, static_cast<uint32_t>(vpp::kTileM)};
+        if (!make_tmap(&tm_q, a->q, 3, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(q) failed");
+    }
+    {
+        const uint64_t d[4] = {static_cast<uint64_t>(a->head_dim_qk), static_cast<uint64_t>(B),
+                               static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
+        const uint64_t s[3] = {static_cast<uint64_t>(a->k_token_stride) * 2, static_cast<uint64_t>(a->k_head_stride) * 2,
+                               static_cast<uint64_t>(a->k_block_stride) * 2};
+        const uint32_t b[4] = {64, static_cast<uint32_t>(box_rows), 1, 1};
+        if (!make_tmap(&tm_k, a->k_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k) failed");
+    }
+    {
+        const uint64_t d[4] = {static_cast<uint64_t>(a->head_dim_v), static_cast<uint64_t>(B),
+                               static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
+        const uint64_t s[3] = {static_cast<uint64_t>(a->v_token_stride) * 2, static_cast<uint64_t>(a->v_head_stride) * 2,
+                               static_cast<uint64_t>(a->v_block_stride) * 2};
+        const uint32_t b[4] = {64, static_cast<uint32_t>(box_rows), 1, 1};
+        if (!make_tmap(&tm_v, a->v_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(v) failed");
+    }
+
+    // ---- work decomposition ----
+    int32_t* row_splits = reinterpret_cast<int32_t*>(ws + L.row_splits);
+    vpp::PrepParams pp{};
+    pp.prefix_len = a->prefix_len;
+    pp.chunk_len = a->chunk_len;
+    pp.block_table = a->block_table;
+    pp.num_reqs = a->num_reqs;
+    pp.total_q = a->total_q;
+    pp.max_seq_len = a->max_seq_len;
+    pp.max_blocks_per_req = a->max_blocks_per_req;
+    pp.block_shift = paged ? ilog2(B) : 0;
+    pp.num_blocks = n_blocks;
+    pp.splits = L.splits;
+    pp.max_units = L.max_units;
+    pp.max_cost = (a->max_seq_len + vpp::kTileN - 1) / vpp::kTileN;
+    if (pp.max_cost < 1) pp.max_cost = 1;
+    pp.header = reinterpret_cast<vpp::WorkHeader*>(ws + L.header);
+    pp.units = reinterpret_cast<vpp::WorkUnit*>(ws + L.units);
+    pp.row_splits = row_splits;
+    pp.q_start = row_splits + a->total_q;
+    pp.tile_start = pp.q_start + a->num_reqs + 1;
+    pp.status = a->status;
+    vpp::prep_kernel<<<1, vpp::kPrepThreads, 0, stream>>>(pp);
+    ++g_launches;
+
+    // ---- attention ----
+    vpp::AttnParams ap{};
+    ap.block_table = a->block_table;
+    ap.max_blocks_per_req = a->max_blocks_per_req;
+    ap.block_shift = pp.block_shift;
+    ap.num_blocks = n_blocks;
+    ap.num_q_heads = a->num_q_heads;
+    ap.num_kv_heads = a->num_kv_heads;
+    ap.total_q = a->total_q;
+    ap.scale_log2e = a->softmax_scale * 1.4426950408889634f;
+    ap.out = a->out;
+    ap.lse = a->lse;
+    ap.o_parts = reinterpret_cast<float*>(ws + L.o_parts);
+    ap.lse_parts = reinterpret_cast<float*>(ws + L.lse_parts);
+    ap.header_ro = pp.header;
+    ap.header = pp.header;
+    ap.units = pp.units;
+    ap.status = a->status;
+
+    const int sms = sm_count_or_default();
+    static const bool p_in_smem = [] {
+        const char* e = std::getenv("VPP_SIMPLE_P_SMEM");
+        return e && e[0] == '1';
+    }();
+    cudaError_t ce;
+    if (p_in_smem) {
+        auto kern = vpp::attn128_simple_kernel<false>;
+        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kSimpleThreads, vpp::kSimpleSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
+    } else {
+        auto kern = vpp::attn128_simple_kernel<true>;
+        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kSimpleThreads, vpp::kSimpleSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
+    }
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "attention kernel attributes: %s", cudaGetErrorString(ce));
+    ++g_launches;
+
+    // ---- merge of split partials ----
+    if (L.splits > 1) {
+        const long long pairs = static_cast<long long>(a->total_q) * a->num_q_heads;
+        const long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+        vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
+            ap.o_parts, ap.lse_parts, L.splits, a->total_q, a->num_q_heads, a->head_dim_v, row_splits,
+            static_cast<__nv_bfloat16*>(a->out), a->lse);
+        ++g_launches;
+    }
+    ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(ce));
+    return VPP_OK;
+}
+
+vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t num_splits, int32_t total_q,
+                         int32_t num_q_heads, int32_t head_dim_v, void* out, float* lse, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    if (num_splits <= 0 || total_q < 0 || num_q_heads <= 0 || head_dim_v <= 0)
+        return fail(VPP_ERR_INVALID_ARG, "num_splits, num_q_heads, head_dim_v must be > 0 and total_q >= 0");
+    if (head_dim_v % 8 != 0) return fail(VPP_ERR_UNSUPPORTED, "head_dim_v must be a multiple of 8");
+    if (total_q == 0) return VPP_OK;
+    if (!o_parts || !lse_parts || !out) return fail(VPP_ERR_INVALID_ARG, "o_parts, lse_parts and out must be non-null");
+    if ((reinterpret_cast<uintptr_t>(o_parts) | reinterpret_cast<uintptr_t>(out)) & 15u)
+        return fail(VPP_ERR_INVALID_ARG, "o_parts and out must be 16-byte aligned");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const long long pairs = static_cast<long long>(total_q) * num_q_heads;
+    const long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+    vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
+        o_parts, lse_parts, num_splits, total_q, num_q_heads, head_dim_v, nullptr, static_cast<__nv_bfloat16*>(out),
+        lse);
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "merge launch: %s", cudaGetErrorString(ce));
+    return VPP_OK;
+}
+
+}  // extern "C"

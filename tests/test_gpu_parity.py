@@ -1,0 +1,98 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_26523_b200 import api, workloads as W
+from parity import compare, run_gpu, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def full_check(prob_cpu, num_kv_splits=0, label=""):
+    out, lse, runner = run_gpu(prob_cpu.to("cuda"), num_kv_splits)
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    return compare(out, lse, prob_cpu, rows, label), runner
+
+
+@pytest.mark.parametrize("k", [0, 1, 2, 3])
+def test_cfg1_every_element(k):
+    s, _ = full_check(W.cfg1(k), label="cfg1 chunk %d" % k)
+    print(s)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 5])
+def test_cfg1_forced_splits(splits):
+    s, _ = full_check(W.cfg1(3), num_kv_splits=splits, label="cfg1 chunk 3 S=%d" % splits)
+    print(s)
+
+
+CASES = [
+    # prefix_lens, chunk_lens, hq, hkv, block_size
+    ([0], [1], 2, 1, None),                       # one token, one key
+    ([0], [129], 4, 2, 128),                      # one row into a second query tile
+    ([127], [2], 2, 2, 64),                       # straddles a KV tile edge
+    ([300], [77], 4, 1, 16),                      # unaligned everything, small pages
+    ([1000, 0, 17, 511], [200, 0, 300, 129], 8, 2, 32),   # varlen batch with an empty request
+    ([4095], [257], 4, 4, 256),                   # pages larger than a KV tile, MHA
+    ([513], [640], 4, 2, None),                   # contiguous cache, several tiles
+    ([0, 0, 0], [5, 130, 1], 2, 1, 128),
+]
+
+
+@pytest.mark.parametrize("case", range(len(CASES)))
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_adversarial_shapes(case, splits):
+    P, C, hq, hkv, bs = CASES[case]
+    prob = W.make_problem(1000 + case, P, C, hq, hkv, 128, 128, block_size=bs)   # NaN tails / unused blocks
+    s, _ = full_check(prob, num_kv_splits=splits, label="case %d S=%d" % (case, splits))
+    print(s)
+
+
+def test_outputs_outside_the_launch_are_untouched():
+    """Canary rows around out / lse keep their value."""
+    prob = W.make_problem(77, [40], [100], 4, 2, 128, 128, block_size=64).to("cuda")
+    big_out = torch.full((102, 4, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    big_lse = torch.full((102, 4), 7.0, dtype=torch.float32, device="cuda")
+    runner = api.ChunkAttn(prob)
+    runner.args.out = big_out[1:].data_ptr()
+    runner.args.lse = big_lse[1:].data_ptr()
+    runner.run()
+    torch.cuda.synchronize()
+    assert (big_out[0] == 7).all() and (big_out[101] == 7).all()
+    assert (big_lse[0] == 7).all() and (big_lse[101] == 7).all()
+    assert torch.isfinite(big_out[1:101].float()).all()
+
+
+def test_lse_merge_against_oracle():
+    g = torch.Generator().manual_seed(5)
+    S, T, Hq, Dv = 5, 37, 3, 128
+    o = torch.randn(S, T, Hq, Dv, generator=g)
+    l = torch.randn(S, T, Hq, generator=g) * 4
+    l[2, 5] = float("-inf")
+    l[:, 7, 1] = float("-inf")
+    out = torch.empty(T, Hq, Dv, dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty(T, Hq, device="cuda")
+    api.vpp_lse_merge(o.cuda(), l.cuda(), out, lse)
+    torch.cuda.synchronize()
+    ro, rl = oracle.ref_lse_merge(o.reshape(S, T * Hq, Dv).double().numpy(), l.reshape(S, T * Hq).double().numpy())
+    got = out.float().cpu().numpy().reshape(T * Hq, Dv)
+    assert np.abs(got - ro).max() <= 2.0 ** -8 * np.abs(ro).max() + 1e-6
+    gl = lse.cpu().numpy().reshape(-1)
+    fin = np.isfinite(rl)
+    assert np.array_equal(np.isneginf(gl), ~fin)
+    assert (np.abs(gl[fin] - rl[fin]) <= 1e-5 * np.maximum(1, np.abs(rl[fin]))).all()
+
+
+def test_bad_lengths_set_device_status_and_write_nothing():
+    prob = W.make_problem(78, [10], [20], 2, 1, 128, 128, block_size=16).to("cuda")
+    runner = api.ChunkAttn(prob)
+    runner.out.fill_(3.0)
+    bad = prob.prefix_len.clone(); bad[0] = 10 ** 6            # beyond max_seq_len
+    runner.args.prefix_len = bad.data_ptr()
+    runner.run()
+    torch.cuda.synchronize()
+    assert int(runner.status.item()) == 1
+    assert (runner.out == 3.0).all()
