@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the chunked-prefill attention path on B200.
+
+A "step" is one pass of the whole hot path (work decomposition -> attention -> merge when split) over
+one batch of synthetic input: the GQA long-context chunk (64 q-heads, 4 kv-heads, head_dim 128, chunk of
+8192 tokens, 128-token pages with a shuffled block table) evaluated once at each of its prefix lengths
+0, 8K, 32K, 64K and 128K.  The reported value is the aggregate TFLOP/s of a step (exact causal flop
+count); the per-prefix latency / TFLOP/s curve -- the cost curve the paper's V-shaped layout is built
+around -- is reported beside it in "curve".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One JSON line on stdout (rank 0).  With --impl reference the CPU oracle is timed on the host cores on a
+bounded sample of the same workload.
+"""
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2608_26523_b200 import workloads as W
+
+METRIC = "chunk-attn TFLOP/s and % dense BF16 peak vs prefix length (1 B200)"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return res
+
+
+def oracle_sample_rate(prob_cpu, target_seconds, rng):
+    """Time the fp64 oracle (as it stands) on random (row, head) samples of the workload.
+
+    Returns (flops done, seconds, rows, threads)."""
+    import oracle
+    C = int(prob_cpu.chunk_len[0]); P = int(prob_cpu.prefix_len[0])
+    hq = prob_cpu.num_q_heads
+    per_row = 2.0 * (prob_cpu.head_dim_qk + prob_cpu.head_dim_v)
+
+    def run(n):
+        rows = np.stack([np.zeros(n, np.int32), rng.integers(0, C, n).astype(np.int32),
+                         rng.integers(0, hq, n).astype(np.int32)], axis=1)
+        t0 = time.perf_counter()
+        oracle.ref_chunk_attn_rows(prob_cpu.q, prob_cpu.k_cache, prob_cpu.v_cache,
+                                   prob_cpu.k_cache.stride()[:3], prob_cpu.v_cache.stride()[:3],
+                                   None if prob_cpu.block_table is None else prob_cpu.block_table.numpy(),
+                                   prob_cpu.block_size, prob_cpu.prefix_len.numpy(), prob_cpu.chunk_len.numpy(),
+                                   hq, prob_cpu.num_kv_heads, prob_cpu.head_dim_qk, prob_cpu.head_dim_v,
+                                   prob_cpu.scale, rows)
+        dt = time.perf_counter() - t0
+        fl = float(((P + rows[:, 1].astype(np.int64) + 1) * per_row).sum())
+        return fl, dt
+
+    threads = oracle.num_threads()
+    fl, dt = run(4 * threads)                       # calibration batch
+    n = int(max(threads, min(4 * threads * target_seconds / max(dt, 1e-3), 200000)))
+    fl, dt = run(n)
+    return fl, dt, n, threads
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--prefixes", default=",".join(str(p) for p in W.CFG2_PREFIXES))
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    prefixes = [int(x) for x in args.prefixes.split(",")]
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    peaks = load_peaks()
+    config = {"workload": "cfg2: GQA Hq=64 Hkv=4 d=128, chunk 8192, prefixes %s, 128-token pages, shuffled block_table"
+              % prefixes, "prefixes": prefixes, "chunk": 8192,
+              "l2": "inputs larger than L2: each step cycles through %d MB of KV plus 134 MB of Q per prefix point"
+              % int((max(prefixes) + 8192) * 4 * 128 * 2 * 2 / 1e6)}
+
+    # ------------------------------------------------------------------------------------------
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        rng = np.random.default_rng(0)
+        budget = 20.0
+        steps_total = args.steps + args.warmup
+        per_step = min(budget, 120.0 / max(steps_total, 1))
+        # a smaller cache is enough for the sample: rows of the 64K point
+        prob = W.cfg2(prefix=65536, device="cpu")
+        times, flops, rows_n = [], [], 0
+        for s in range(steps_total):
+            fl, dt, n, threads = oracle_sample_rate(prob, per_step, rng)
+            if s >= args.warmup:
+                times.append(dt); flops.append(fl); rows_n += n
+        val = sum(flops) / sum(times) / 1e12
+        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(times) / len(times),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                 "sample": "%d random (row, head) pairs of the chunk at prefix 65536 over %d steps"
+                                 % (rows_n, args.steps)},
+                "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line), flush=True)
+        return
+
+    # ------------------------------------------------------------------------------------------
+    from paper_2608_26523_b200 import api
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    api.load_library()
+
+    max_prefix = max(prefixes)
+    base = W.cfg2(prefix=max_prefix, max_prefix=max_prefix, device=dev)
+    stream = torch.cuda.Stream(device=dev)
+    runners = []
+    for P in prefixes:
+        prob = base.with_chunk([P], [8192], base.q)
+        runners.append(api.ChunkAttn(prob, num_kv_splits=args.splits))
+    flops_pt = [r.prob.flops() for r in runners]
+    flops_step = float(sum(flops_pt))
+    launches_per_step = 0
+
+    def one_step(events=None):
+        for i, r in enumerate(runners):
+            if events is not None:
+                events[i][0].record(stream)
+            r.run(stream.cuda_stream)
+            if events is not None:
+                events[i][1].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            one_step()
+        launches_per_step = 0
+        for r in runners:
+            r.run(stream.cuda_stream)
+            launches_per_step += api.vpp_last_launch_count()
+        barrier()
+        for r in runners:
+            assert int(r.status.item()) == 0, "device status %d" % int(r.status.item())
+
+        sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sampler.start()
+            time.sleep(0.3)
+        ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in runners]
+              for _ in range(args.steps)]
+        t_beg = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+        barrier()
+        t_beg.record(stream)
+        for s in range(args.steps):
+            one_step(ev[s])
+        t_end.record(stream)
+        barrier()
+        clocks = sampler.stop() if rank == 0 else None
+        total_ms = t_beg.elapsed_time(t_end)
+        per_pt_ms = [statistics.median(ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps))
+                     for i in range(len(runners))]
+
+        # ---- end to end: host buffers in, host buffers out, copies inside the timed region ----
+        e2e = None
+        if not args.no_e2e:
+            i_main = prefixes.index(65536) if 65536 in prefixes else len(prefixes) - 1
+            r = runners[i_main]
+            P = prefixes[i_main]
+            q_host = r.prob.q.cpu().pin_memory()
+            out_host = torch.empty(r.out.shape, dtype=r.out.dtype).pin_memory()
+            lse_host = torch.empty(r.lse.shape, dtype=r.lse.dtype).pin_memory()
+            bt = r.prob.block_table[0].cpu().tolist()
+            B = r.prob.block_size
+            chunk_blocks = [bt[j] for j in range(P // B, (P + 8192 + B - 1) // B)]
+            k_host = [r.prob.k_cache[b].cpu().pin_memory() for b in chunk_blocks]
+            v_host = [r.prob.v_cache[b].cpu().pin_memory() for b in chunk_blocks]
+            h2d = q_host.numel() * 2 + sum(t.numel() * 2 for t in k_host + v_host)
+            d2h = out_host.numel() * 2 + lse_host.numel() * 4
+
+            def e2e_step():
+                r.prob.q.copy_(q_host, non_blocking=True)
+                for b, kh, vh in zip(chunk_blocks, k_host, v_host):   # the chunk's own K/V pages
+                    r.prob.k_cache[b].copy_(kh, non_blocking=True)
+                    r.prob.v_cache[b].copy_(vh, non_blocking=True)
+                r.run(stream.cuda_stream)
+                out_host.copy_(r.out, non_blocking=True)
+                lse_host.copy_(r.lse, non_blocking=True)
+
+            for _ in range(2):
+                e2e_step()
+            barrier()
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            n_e2e = max(args.steps, 3)
+            for _ in range(n_e2e):
+                e2e_step()
+            t1.record(stream)
+            barrier()
+            e2e_ms = t0.elapsed_time(t1) / n_e2e
+            e2e = (flops_pt[i_main], e2e_ms, h2d, d2h, P)
+
+    # ---- max over ranks ----
+    if world > 1:
+        t = torch.tensor([total_ms, e2e[1] if e2e else 0.0], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t[0])
+        if e2e:
+            e2e = (e2e[0], float(t[1]), e2e[2], e2e[3], e2e[4])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = total_ms / args.steps
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    burst, sustained = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    curve = []
+    for P, ms, fl in zip(prefixes, per_pt_ms, flops_pt):
+        tf = fl / (ms * 1e-3) / 1e12
+        curve.append({"prefix": P, "ms": round(ms, 4), "tflops": round(tf, 2), "frac_of_burst_peak": round(tf / burst, 4),
+                      "frac_of_sustained_peak": round(tf / sustained, 4)})
+    # dominant kernel = the attention kernel at the longest prefix; its launch is timed together with the
+    # ~10 us work-decomposition kernel that precedes it on the same stream
+    i_top = int(np.argmax(flops_pt))
+    ach = flops_pt[i_top] / (per_pt_ms[i_top] * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": round(ach, 2), "peak": burst, "unit": "TFLOP/s",
+                "frac": round(ach / burst, 4), "traffic": None, "peak_source": "%s (burst bf16 matmul)" % peaks["_source"],
+                "frac_of_sustained": round(ach / sustained, 4), "kernel": "attention kernel, prefix %d" % prefixes[i_top]}
+    line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config, "curve": curve,
+            "roofline": roofline, "gpu_launches": launches_per_step * args.steps, "clocks": clocks}
+    if e2e:
+        line["e2e"] = {"value": round(world * e2e[0] / (e2e[1] * 1e-3) / 1e12, 3), "unit": UNIT,
+                       "h2d_bytes_per_step": int(e2e[2]), "d2h_bytes_per_step": int(e2e[3]),
+                       "ms_per_step": round(e2e[1], 4),
+                       "workload": "the chunk at prefix %d: q and the chunk's K/V pages host->device, out and lse device->host" % e2e[4]}
+    if not args.no_cpu_baseline and world == 1:
+        prob_cpu = runners[prefixes.index(65536) if 65536 in prefixes else -1].prob.to("cpu")
+        fl, dt, n, threads = oracle_sample_rate(prob_cpu, 15.0, np.random.default_rng(0))
+        line["cpu_baseline"] = {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": "%d random (row, head) pairs of the chunk at prefix %d (%.1f s of CPU time)"
+                                % (n, int(prob_cpu.prefix_len[0]), dt)}
+    if world > 1:
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -12,6 +12,7 @@
 
 #include "../../include/vpp.h"
 #include "attn_simple.cuh"
+#include "attn_ws.cuh"
 #include "common.cuh"
 #include "merge.cuh"
 #include "prep.cuh"
@@ -166,7 +167,20 @@ int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
     return static_cast<int>(s);
 }
 
-int heads_per_item(const vpp_chunk_attn_args*, Family) { return 1; }
+// The pipelined kernel pairs two q-heads of one kv-head per work item; odd group sizes (MHA) take the
+// straight-line kernel, one head per item.  VPP_FORCE_SIMPLE=1 selects the straight-line kernel always
+// (a debugging aid; read once).
+bool force_simple() {
+    static const bool v = [] {
+        const char* e = std::getenv("VPP_FORCE_SIMPLE");
+        return e && e[0] == '1';
+    }();
+    return v;
+}
+bool use_ws_kernel(const vpp_chunk_attn_args* a) {
+    return !force_simple() && ((a->num_q_heads / a->num_kv_heads) % 2 == 0);
+}
+int heads_per_item(const vpp_chunk_attn_args* a, Family) { return use_ws_kernel(a) ? 2 : 1; }
 
 vpp::WorkspaceLayout layout_for(const vpp_chunk_attn_args* a, Family fam) {
     vpp::WorkspaceLayout L{};
@@ -316,15 +330,11 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     ap.status = a->status;
 
     const int sms = sm_count_or_default();
-    static const bool p_in_smem = [] {
-        const char* e = std::getenv("VPP_SIMPLE_P_SMEM");
-        return e && e[0] == '1';
-    }();
     cudaError_t ce;
-    if (p_in_smem) {
-        auto kern = vpp::attn128_simple_kernel<false>;
-        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kSimpleThreads, vpp::kSimpleSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
+    if (use_ws_kernel(a)) {
+        auto kern = vpp::attn128_ws_kernel;
+        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
     } else {
         auto kern = vpp::attn128_simple_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);

@@ -1,0 +1,471 @@
+// Warp-specialised persistent chunked-prefill attention kernel for head_dim 128 (GQA / MQA with an
+// even group size).
+//
+// One CTA per SM, 12 warps:
+//   warp 0      scheduler + TMA producer: pops work items from the global counter, publishes them in a
+//               2-deep shared ring, loads the two Q tiles of the item and streams K/V pages through a
+//               ring of 128B-swizzled 32 KB stages (K0 V0 K1 V1 ...), gathered through the block table.
+//   warp 1      MMA issuer: tcgen05.mma  S_t = Q_t K^T  and  O_t += P_t V  for the two query tiles
+//               t = 0, 1 of the item (two q-heads of one kv-head over the same 128 query tokens, so
+//               both tiles use the same K/V stages and the same causal structure).
+//   warp 2      tensor-memory allocation.
+//   warps 4-7   softmax group for tile 0: one query row per thread, fp32 online softmax on S_0 read
+//               from tensor memory, P_0 written back to tensor memory as bf16 over S_0.
+//   warps 8-11  the same for tile 1.
+// While one group works on its S tile the tensor core runs the other tile's MMAs.
+// Tensor memory: S_0 | S_1 | O_0 | O_1, 128 fp32 columns each (all 512 columns).
+//
+// The math per row is the paper's Eq. 1 with the causal rule, evaluated KV tile by KV tile with a
+// running maximum; O is rescaled lazily (only when the maximum has grown by more than 2^8).
+#pragma once
+#include "attn_simple.cuh"  // decode_item, kSlabBytes
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace vpp {
+
+constexpr int kWsThreads = 384;
+constexpr int kWsStages = 4;                  // 32 KB each
+constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
+constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 1024 /*barriers, ring*/;
+constexpr float kRescaleThreshold = 8.f;      // log2 units
+
+struct WsItem {
+    WorkUnit u;
+    int32_t h0;     // first of the two q-heads
+    int32_t valid;  // 0: no more work
+    int32_t pad[2];
+};
+
+__device__ __forceinline__ void setmaxnreg_dec56() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
+__device__ __forceinline__ void setmaxnreg_inc224() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
+
+__global__ void __launch_bounds__(kWsThreads, 1)
+attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p, const int kv_box_rows) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sQ = smem_base;                       // 2 tiles
+    const uint32_t sKV = sQ + 2 * kTileBytes;            // kWsStages tiles
+    const uint32_t sBar = sKV + kWsStages * kTileBytes;  // barriers
+    // barrier map (8 bytes each)
+    const uint32_t bar_item_full = sBar + 0;     // [2]
+    const uint32_t bar_item_empty = sBar + 16;   // [2]
+    const uint32_t bar_q_full = sBar + 32;
+    const uint32_t bar_q_empty = sBar + 40;
+    const uint32_t bar_s_full = sBar + 48;       // [2]
+    const uint32_t bar_p_full = sBar + 64;       // [2]
+    const uint32_t bar_o_full = sBar + 80;       // [2]
+    const uint32_t bar_vfix = sBar + 96;
+    const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
+    const uint32_t bar_kv_empty = sBar + 128 + 8 * kWsStages;
+    uint8_t* gen_bar = gen_base + (2 + kWsStages) * kTileBytes;
+    volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 512);
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 516);
+    WsItem* ring = reinterpret_cast<WsItem*>(gen_bar + 576);  // 2 x 48 bytes
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    if (tid == 0) {
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar_item_full + 8 * i, 1);
+            mbar_init(bar_item_empty + 8 * i, 9);
+            mbar_init(bar_s_full + 8 * i, 1);
+            mbar_init(bar_p_full + 8 * i, 128);
+            mbar_init(bar_o_full + 8 * i, 1);
+        }
+        mbar_init(bar_q_full, 1);
+        mbar_init(bar_q_empty, 1);
+        mbar_init(bar_vfix, 1);
+        for (int i = 0; i < kWsStages; ++i) {
+            mbar_init(bar_kv_full + 8 * i, 1);
+            mbar_init(bar_kv_empty + 8 * i, 1);
+        }
+        fence_mbar_init();
+        *s_abort = 0;
+        prefetch_tmap(&tm_q);
+        prefetch_tmap(&tm_k);
+        prefetch_tmap(&tm_v);
+    }
+    __syncthreads();
+    if (warp == 2) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(s_tmem)), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    const int num_units = p.header_ro->num_units;
+    const int G = p.num_q_heads / p.num_kv_heads;
+    const int total_items = num_units * (p.num_q_heads / 2);
+
+    if (warp < 4) {
+        setmaxnreg_dec56();
+        if (warp == 0) {
+            // ============================ scheduler + TMA producer ============================
+            uint32_t item_it = 0, q_it = 0, kv_it = 0;
+            while (true) {
+                int item = 0;
+                if (lane == 0) item = atomicAdd(&p.header->counter, 1);
+                item = __shfl_sync(0xffffffffu, item, 0);
+                const bool have = item < total_items;
+                const uint32_t slot = item_it & 1;
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(bar_item_empty + 8 * slot, ((item_it >> 1) & 1) ^ 1, s_abort, 201);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                WorkUnit u{};
+                int h0 = 0;
+                if (have) {
+                    int ui, hp;
+                    decode_item(item, num_units, p.num_q_heads / 2, G / 2, ui, hp);
+                    u = p.units[ui];
+                    h0 = 2 * hp;
+                }
+                if (lane == 0) {
+                    ring[slot].u = u;
+                    ring[slot].h0 = h0;
+                    ring[slot].valid = have ? 1 : 0;
+                    mbar_arrive(bar_item_full + 8 * slot);
+                }
+                ++item_it;
+                if (!have) break;
+                const int g = h0 / G;
+
+                if (lane == 0) {
+                    ok = mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 202);
+                    if (ok) {
+                        mbar_arrive_expect_tx(bar_q_full, 2 * kTileBytes);
+                        tma_load_3d(sQ, &tm_q, bar_q_full, 0, h0, u.q_row0);
+                        tma_load_3d(sQ + kSlabBytes, &tm_q, bar_q_full, 64, h0, u.q_row0);
+                        tma_load_3d(sQ + kTileBytes, &tm_q, bar_q_full, 0, h0 + 1, u.q_row0);
+                        tma_load_3d(sQ + kTileBytes + kSlabBytes, &tm_q, bar_q_full, 64, h0 + 1, u.q_row0);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                ++q_it;
+
+                for (int j = u.kv_begin; j < u.kv_end && ok; ++j) {
+                    const int tile0 = j * kTileN;
+#pragma unroll
+                    for (int which = 0; which < 2; ++which) {  // 0: K, 1: V
+                        const uint32_t st = kv_it % kWsStages;
+                        const uint32_t ph = (kv_it / kWsStages) & 1;
+                        const uint32_t dst = sKV + st * kTileBytes;
+                        const uint32_t full = bar_kv_full + 8 * st;
+                        if (lane == 0) {
+                            ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
+                            if (ok) {
+                                mbar_arrive_expect_tx(full, kTileBytes);
+                                const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+                                for (int off = 0; off < kTileN; off += kv_box_rows) {
+                                    const int pos = tile0 + off;
+                                    int blk, slot_in;
+                                    if (p.block_table == nullptr) {
+                                        blk = u.req;
+                                        slot_in = pos;
+                                    } else if (pos < u.kv_len) {
+                                        blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                                    (pos >> p.block_shift));
+                                        slot_in = pos & ((1 << p.block_shift) - 1);
+                                    } else {
+                                        blk = p.num_blocks;  // out of range: the copy engine fills zeros
+                                        slot_in = 0;
+                                    }
+                                    const uint32_t o = static_cast<uint32_t>(off) * 128u;
+                                    tma_load_4d(dst + o, tm, full, 0, slot_in, g, blk);
+                                    tma_load_4d(dst + kSlabBytes + o, tm, full, 64, slot_in, g, blk);
+                                }
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) break;
+                        if (which == 1 && tile0 + kTileN > u.kv_len) {
+                            // Keys at or beyond kv_len do not exist; zero their V rows so that 0 * garbage
+                            // cannot poison O.  The MMA warp waits for bar_vfix on such a tile.
+                            if (lane == 0) ok = mbar_wait(full, ph, s_abort, 204);
+                            ok = __shfl_sync(0xffffffffu, ok, 0);
+                            if (!ok) break;
+                            uint8_t* vb = gen_base + 2 * kTileBytes + st * kTileBytes;
+                            const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
+                            const uint4 z = make_uint4(0, 0, 0, 0);
+                            for (int r = first + lane; r < kTileN; r += 32) {
+                                uint4* a = reinterpret_cast<uint4*>(vb + r * 128);
+                                uint4* b = reinterpret_cast<uint4*>(vb + kSlabBytes + r * 128);
+#pragma unroll
+                                for (int c = 0; c < 8; ++c) {
+                                    a[c] = z;
+                                    b[c] = z;
+                                }
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_vfix);
+                        }
+                        ++kv_it;
+                    }
+                }
+                if (!ok) break;
+            }
+        } else if (warp == 1) {
+            // ==================================== MMA issuer ====================================
+            constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
+            constexpr uint32_t kIdescPV = idesc_bf16(128, 128, false, true);
+            const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128, tO0 = tmem_base + 256, tO1 = tmem_base + 384;
+            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0;
+            auto wait1 = [&](uint32_t bar, uint32_t parity, int where) -> bool {
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(bar, parity, s_abort, where);
+                return __shfl_sync(0xffffffffu, ok, 0);
+            };
+            auto issue_qk = [&](uint32_t tS, uint32_t q_tile, uint32_t k_stage) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t koff = (k >> 2) * kSlabBytes + (k & 3) * 32;
+                    mma_ss(tS, smem_desc_sw128(q_tile + koff, 16, 1024), smem_desc_sw128(k_stage + koff, 16, 1024),
+                           kIdescQK, k > 0);
+                }
+            };
+            auto issue_pv = [&](uint32_t tO, uint32_t tP, uint32_t v_stage, bool first) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    mma_ts(tO, tP + k * 8, smem_desc_sw128(v_stage + k * 2048, kSlabBytes, 1024), kIdescPV,
+                           (!first || k > 0) ? 1u : 0u);
+            };
+            while (true) {
+                const uint32_t slot = item_it & 1;
+                if (!wait1(bar_item_full + 8 * slot, (item_it >> 1) & 1, 301)) break;
+                const WorkUnit u = ring[slot].u;
+                const int valid = ring[slot].valid;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
+                ++item_it;
+                if (!valid) break;
+                const int n = u.kv_end - u.kv_begin;
+                if (!wait1(bar_q_full, q_it & 1, 302)) break;
+                ++q_it;
+                // S_t(0) = Q_t K(0)^T
+                uint32_t stK = kv_it % kWsStages;
+                if (!wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 303)) break;
+                ++kv_it;
+                tc_fence_after();
+                if (lane == 0) {
+                    issue_qk(tS0, sQ, sKV + stK * kTileBytes);
+                    tc_commit(bar_s_full);
+                    issue_qk(tS1, sQ + kTileBytes, sKV + stK * kTileBytes);
+                    tc_commit(bar_s_full + 8);
+                    tc_commit(bar_kv_empty + 8 * stK);
+                    if (n == 1) tc_commit(bar_q_empty);
+                }
+                bool ok = true;
+                for (int jj = 0; jj < n && ok; ++jj) {
+                    const int tile0 = (u.kv_begin + jj) * kTileN;
+                    const uint32_t stV = kv_it % kWsStages;
+                    ok = wait1(bar_kv_full + 8 * stV, (kv_it / kWsStages) & 1, 304);
+                    if (!ok) break;
+                    ++kv_it;
+                    if (tile0 + kTileN > u.kv_len) {
+                        ok = wait1(bar_vfix, vfix_it & 1, 305);
+                        if (!ok) break;
+                        ++vfix_it;
+                    }
+                    const bool has_next = jj + 1 < n;
+                    stK = kv_it % kWsStages;
+                    // ---- tile 0 ----
+                    ok = wait1(bar_p_full, p_it & 1, 306);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0);
+                    if (has_next) {
+                        ok = wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 307);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (lane == 0) {
+                            issue_qk(tS0, sQ, sKV + stK * kTileBytes);
+                            tc_commit(bar_s_full);
+                        }
+                    } else if (lane == 0) {
+                        tc_commit(bar_o_full);
+                    }
+                    // ---- tile 1 ----
+                    ok = wait1(bar_p_full + 8, p_it & 1, 308);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0);
+                        tc_commit(bar_kv_empty + 8 * stV);
+                        if (has_next) {
+                            issue_qk(tS1, sQ + kTileBytes, sKV + stK * kTileBytes);
+                            tc_commit(bar_s_full + 8);
+                            tc_commit(bar_kv_empty + 8 * stK);
+                            if (jj + 2 == n) tc_commit(bar_q_empty);
+                        } else {
+                            tc_commit(bar_o_full + 8);
+                        }
+                    }
+                    if (has_next) ++kv_it;
+                    ++p_it;
+                }
+                if (!ok) break;
+            }
+        }
+        // warps 2 and 3 have nothing to do until teardown
+    } else {
+        // ===================================== softmax groups =====================================
+        setmaxnreg_inc224();
+        const int t = (warp - 4) >> 2;                 // query tile / softmax group
+        const int row = ((warp & 3) << 5) | lane;      // row of the tile = TMEM lane
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + t * 128 + lane_off;
+        const uint32_t tO = tmem_base + 256 + t * 128 + lane_off;
+        const uint32_t bar_s = bar_s_full + 8 * t, bar_p = bar_p_full + 8 * t, bar_o = bar_o_full + 8 * t;
+        uint32_t item_it = 0, s_it = 0, o_it = 0;
+        const float sc = p.scale_log2e;
+        while (true) {
+            const uint32_t slot = item_it & 1;
+            if (!mbar_wait(bar_item_full + 8 * slot, (item_it >> 1) & 1, s_abort, 401)) break;
+            const WorkUnit u = ring[slot].u;
+            const int h = ring[slot].h0 + t;
+            const int valid = ring[slot].valid;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
+            ++item_it;
+            if (!valid) break;
+
+            const int my_pos = u.pos0 + row;
+            float m_ref = -INFINITY, l_run = 0.f;
+            bool ok = true;
+            for (int j = u.kv_begin; j < u.kv_end; ++j) {
+                const int tile0 = j * kTileN;
+                ok = mbar_wait(bar_s, s_it & 1, s_abort, 402);
+                if (!ok) break;
+                ++s_it;
+                tc_fence_after();
+                uint32_t s[128];
+                tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
+                tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
+                tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(s[64]));
+                tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(s[96]));
+                tc_wait_ld();
+                if (tile0 + kTileN - 1 > u.pos0) {  // diagonal tile: keys beyond the row's position are masked
+                    const int lim = my_pos - tile0;  // columns <= lim are visible
+#pragma unroll
+                    for (int i = 0; i < 128; ++i)
+                        if (i > lim) s[i] = 0xff800000u;  // -inf
+                }
+                float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
+#pragma unroll
+                for (int i = 2; i < 128; i += 2) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[i]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[i + 1]));
+                }
+                const float m_new = fmaxf(fmaxf(mx0, mx1) * sc, m_ref);
+                // lazy rescale: keep the old reference unless the maximum moved by more than 2^8
+                const bool grow = (m_new - m_ref > kRescaleThreshold) || (m_ref == -INFINITY && m_new != -INFINITY);
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float alpha = grow ? ex2(m_ref - m_new) : 1.f;  // m_ref = -inf gives 0
+                    if (grow) m_ref = m_new;
+                    l_run *= alpha;
+                    if (j > u.kv_begin) {
+                        uint32_t o[32];
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            tmem_ld32(tO + c * 32, o);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                    }
+                }
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use));
+                        const float p1 = ex2(fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use));
+                        sum0 += p0;
+                        sum1 += p1;
+                        pk[i >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                l_run += sum0 + sum1;
+                tc_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar_p);
+            }
+            if (!ok) break;
+
+            // ---- epilogue ----
+            ok = mbar_wait(bar_o, o_it & 1, s_abort, 403);
+            if (!ok) break;
+            ++o_it;
+            tc_fence_after();
+            {
+                const float inv_l = 1.f / l_run;
+                const bool live = row < u.rows;
+                const long long grow_idx = static_cast<long long>(u.q_row0) + row;
+                uint32_t r[32];
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    tmem_ld32(tO + c * 32, r);
+                    tc_wait_ld();
+                    if (!live) continue;
+                    if (u.split < 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                              ((grow_idx * p.num_q_heads + h) * 128 + c * 32) * 2);
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                w[e] = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2 * e]) * inv_l,
+                                                   __uint_as_float(r[q4 * 8 + 2 * e + 1]) * inv_l);
+                            dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(
+                            p.o_parts +
+                            ((static_cast<long long>(u.split) * p.total_q + grow_idx) * p.num_q_heads + h) * 128 + c * 32);
+#pragma unroll
+                        for (int q4 = 0; q4 < 8; ++q4)
+                            dst[q4] = make_float4(__uint_as_float(r[q4 * 4]) * inv_l, __uint_as_float(r[q4 * 4 + 1]) * inv_l,
+                                                  __uint_as_float(r[q4 * 4 + 2]) * inv_l,
+                                                  __uint_as_float(r[q4 * 4 + 3]) * inv_l);
+                    }
+                }
+                if (live) {
+                    const float lse = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+                    if (u.split < 0) {
+                        if (p.lse) p.lse[grow_idx * p.num_q_heads + h] = lse;
+                    } else {
+                        p.lse_parts[(static_cast<long long>(u.split) * p.total_q + grow_idx) * p.num_q_heads + h] = lse;
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+    }
+
+    // ---- teardown ----
+    __syncthreads();
+    if (*s_abort != 0) {
+        if (tid == 0 && p.status) atomicCAS(p.status, 0, 3 /* VPP_DEV_TIMEOUT */);
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);  // let copies and MMAs in flight drain
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 2) tmem_dealloc(tmem_base, 512);
+}
+
+}  // namespace vpp
