@@ -34,6 +34,7 @@ def build(force=False, verbose=False):
            "-Xcompiler", "-fPIC", "-shared", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("VPP_NVCC_FLAGS", "").split()
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

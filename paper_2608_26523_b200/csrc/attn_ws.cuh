@@ -55,7 +55,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_q_full = sBar + 32;
     const uint32_t bar_q_empty = sBar + 40;
     const uint32_t bar_s_full = sBar + 48;       // [2]
-    const uint32_t bar_p_full = sBar + 64;       // [2]
+    const uint32_t bar_p_full = sBar + 64;       // [2 tiles] (first half of P)
+    const uint32_t bar_p_full_b = sBar + 104;    // [2 tiles] (second half of P)
     const uint32_t bar_o_full = sBar + 80;       // [2]
     const uint32_t bar_vfix = sBar + 96;
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
@@ -75,6 +76,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(bar_item_empty + 8 * i, 9);
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_p_full + 8 * i, 128);
+            mbar_init(bar_p_full_b + 8 * i, 128);
             mbar_init(bar_o_full + 8 * i, 1);
         }
         mbar_init(bar_q_full, 1);
@@ -224,19 +226,23 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (lane == 0) ok = mbar_wait(bar, parity, s_abort, where);
                 return __shfl_sync(0xffffffffu, ok, 0);
             };
-            auto issue_qk = [&](uint32_t tS, uint32_t q_tile, uint32_t k_stage) {
+            // Descriptors are advanced by adding constants to their low word: the single issuing thread
+            // must not spend longer building operands than the tensor core spends on the MMA.
+            constexpr uint32_t kHi = desc_hi_sw128(1024);
+            const uint32_t q_lo0 = desc_lo_sw128(sQ, 16), q_lo1 = desc_lo_sw128(sQ + kTileBytes, 16);
+            auto issue_qk = [&](uint32_t tS, uint32_t q_lo, uint32_t k_stage) {
+                const uint32_t k_lo = desc_lo_sw128(k_stage, 16);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
-                    const uint32_t koff = (k >> 2) * kSlabBytes + (k & 3) * 32;
-                    mma_ss(tS, smem_desc_sw128(q_tile + koff, 16, 1024), smem_desc_sw128(k_stage + koff, 16, 1024),
-                           kIdescQK, k > 0);
+                    const uint32_t koff = ((k >> 2) * kSlabBytes + (k & 3) * 32) >> 4;
+                    mma_ss_lh(tS, q_lo + koff, k_lo + koff, kHi, kIdescQK, k > 0);
                 }
             };
-            auto issue_pv = [&](uint32_t tO, uint32_t tP, uint32_t v_stage, bool first) {
+            auto issue_pv = [&](uint32_t tO, uint32_t tP, uint32_t v_stage, bool first, int k0, int k1) {
+                const uint32_t v_lo = desc_lo_sw128(v_stage, kSlabBytes);
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    mma_ts(tO, tP + k * 8, smem_desc_sw128(v_stage + k * 2048, kSlabBytes, 1024), kIdescPV,
-                           (!first || k > 0) ? 1u : 0u);
+                for (int k = k0; k < k1; ++k)
+                    mma_ts_lh(tO, tP + k * 8, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
             };
             while (true) {
                 const uint32_t slot = item_it & 1;
@@ -256,9 +262,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 ++kv_it;
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_qk(tS0, sQ, sKV + stK * kTileBytes);
+                    issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                     tc_commit(bar_s_full);
-                    issue_qk(tS1, sQ + kTileBytes, sKV + stK * kTileBytes);
+                    issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
                     tc_commit(bar_s_full + 8);
                     tc_commit(bar_kv_empty + 8 * stK);
                     if (n == 1) tc_commit(bar_q_empty);
@@ -281,13 +287,21 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_p_full, p_it & 1, 306);
                     if (!ok) break;
                     tc_fence_after();
-                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0);
+#ifdef VPP_SPLIT_P
+                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 4);
+                    ok = wait1(bar_p_full_b, p_it & 1, 309);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 4, 8);
+#else
+                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
+#endif
                     if (has_next) {
                         ok = wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 307);
                         if (!ok) break;
                         tc_fence_after();
                         if (lane == 0) {
-                            issue_qk(tS0, sQ, sKV + stK * kTileBytes);
+                            issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                             tc_commit(bar_s_full);
                         }
                     } else if (lane == 0) {
@@ -297,11 +311,21 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_p_full + 8, p_it & 1, 308);
                     if (!ok) break;
                     tc_fence_after();
+#ifdef VPP_SPLIT_P
+                    if (lane == 0) issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 4);
+                    ok = wait1(bar_p_full_b + 8, p_it & 1, 310);
+                    if (!ok) break;
+                    tc_fence_after();
+#endif
                     if (lane == 0) {
-                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0);
+#ifdef VPP_SPLIT_P
+                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 4, 8);
+#else
+                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 8);
+#endif
                         tc_commit(bar_kv_empty + 8 * stV);
                         if (has_next) {
-                            issue_qk(tS1, sQ + kTileBytes, sKV + stK * kTileBytes);
+                            issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
                             tc_commit(bar_s_full + 8);
                             tc_commit(bar_kv_empty + 8 * stK);
                             if (jj + 2 == n) tc_commit(bar_q_empty);
@@ -325,6 +349,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint32_t tS = tmem_base + t * 128 + lane_off;
         const uint32_t tO = tmem_base + 256 + t * 128 + lane_off;
         const uint32_t bar_s = bar_s_full + 8 * t, bar_p = bar_p_full + 8 * t, bar_o = bar_o_full + 8 * t;
+        const uint32_t bar_pb = bar_p_full_b + 8 * t;
         uint32_t item_it = 0, s_it = 0, o_it = 0;
         const float sc = p.scale_log2e;
         while (true) {
@@ -359,13 +384,16 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int i = 0; i < 128; ++i)
                         if (i > lim) s[i] = 0xff800000u;  // -inf
                 }
-                float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]);
+                float mx[8];
 #pragma unroll
-                for (int i = 2; i < 128; i += 2) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[i]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[i + 1]));
-                }
-                const float m_new = fmaxf(fmaxf(mx0, mx1) * sc, m_ref);
+                for (int k = 0; k < 8; ++k) mx[k] = __uint_as_float(s[k]);
+#pragma unroll
+                for (int i = 8; i < 128; i += 8)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) mx[k] = fmaxf(mx[k], __uint_as_float(s[i + k]));
+                const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                        fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                const float m_new = fmaxf(mxa * sc, m_ref);
                 // lazy rescale: keep the old reference unless the maximum moved by more than 2^8
                 const bool grow = (m_new - m_ref > kRescaleThreshold) || (m_ref == -INFINITY && m_new != -INFINITY);
                 if (__any_sync(0xffffffffu, grow)) {
@@ -391,18 +419,34 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
+#ifdef VPP_EXP_FAKE  // timing experiment only: results are wrong
+                        const float p0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
+                        const float p1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
+#else
                         const float p0 = ex2(fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use));
                         const float p1 = ex2(fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use));
+#endif
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(tS + c * 16, pk);
+#ifdef VPP_SPLIT_P
+                    if (c == 1) {  // first 64 keys of P are in place: the MMA warp may start O += P V on them
+                        tc_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar_p);
+                    }
+#endif
                 }
                 l_run += sum0 + sum1;
                 tc_wait_st();
                 tc_fence_before();
+#ifdef VPP_SPLIT_P
+                mbar_arrive(bar_pb);
+#else
                 mbar_arrive(bar_p);
+#endif
             }
             if (!ok) break;
 
