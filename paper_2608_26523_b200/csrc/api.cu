@@ -378,4 +378,11 @@ vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t n
     return VPP_OK;
 }
 
+#ifdef VPP_TRACE
+// Timing experiment only: copies the clock stamps of CTA 0 to the host (synchronises).
+int vpp_debug_trace(long long* host_out, int n) {
+    return static_cast<int>(cudaMemcpyFromSymbol(host_out, vpp::g_trace, sizeof(long long) * n));
+}
+#endif
+
 }  // extern "C"

@@ -25,10 +25,24 @@
 namespace vpp {
 
 constexpr int kWsThreads = 384;
-constexpr int kWsStages = 4;                  // 32 KB each
+#ifndef VPP_WS_STAGES
+#define VPP_WS_STAGES 4
+#endif
+constexpr int kWsStages = VPP_WS_STAGES;      // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 1024 /*barriers, ring*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
+
+#ifdef VPP_TRACE
+// Timing experiment only (never part of the product build): clock64 stamps of CTA 0's roles.
+__device__ long long g_trace[64 * 32];
+#define VPP_TR(role, jj, k)                                                                     \
+    do {                                                                                        \
+        if (blockIdx.x == 0 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
+    } while (0)
+#else
+#define VPP_TR(role, jj, k) do {} while (0)
+#endif
 
 struct WsItem {
     WorkUnit u;
@@ -162,7 +176,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         const uint32_t dst = sKV + st * kTileBytes;
                         const uint32_t full = bar_kv_full + 8 * st;
                         if (lane == 0) {
+                            VPP_TR(3, j - u.kv_begin, which * 3 + 0);
                             ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
+                            VPP_TR(3, j - u.kv_begin, which * 3 + 1);
                             if (ok) {
                                 mbar_arrive_expect_tx(full, kTileBytes);
                                 const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
@@ -184,6 +200,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                     tma_load_4d(dst + o, tm, full, 0, slot_in, g, blk);
                                     tma_load_4d(dst + kSlabBytes + o, tm, full, 64, slot_in, g, blk);
                                 }
+                                VPP_TR(3, j - u.kv_begin, which * 3 + 2);
                             }
                         }
                         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -215,22 +232,23 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
                 if (!ok) break;
             }
-        } else if (warp == 1) {
-            // ==================================== MMA issuer ====================================
+        } else if (warp == 1 && lane == 0) {
+            // ============================ MMA issuer (a single thread) ============================
             constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
             constexpr uint32_t kIdescPV = idesc_bf16(128, 128, false, true);
             const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128, tO0 = tmem_base + 256, tO1 = tmem_base + 384;
             uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0;
             auto wait1 = [&](uint32_t bar, uint32_t parity, int where) -> bool {
-                bool ok = true;
-                if (lane == 0) ok = mbar_wait(bar, parity, s_abort, where);
-                return __shfl_sync(0xffffffffu, ok, 0);
+                return mbar_wait(bar, parity, s_abort, where);
             };
             // Descriptors are advanced by adding constants to their low word: the single issuing thread
             // must not spend longer building operands than the tensor core spends on the MMA.
             constexpr uint32_t kHi = desc_hi_sw128(1024);
             const uint32_t q_lo0 = desc_lo_sw128(sQ, 16), q_lo1 = desc_lo_sw128(sQ + kTileBytes, 16);
             auto issue_qk = [&](uint32_t tS, uint32_t q_lo, uint32_t k_stage) {
+#ifdef VPP_T_NO_QK
+                return;
+#endif
                 const uint32_t k_lo = desc_lo_sw128(k_stage, 16);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
@@ -239,18 +257,29 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             };
             auto issue_pv = [&](uint32_t tO, uint32_t tP, uint32_t v_stage, bool first, int k0, int k1) {
+#ifdef VPP_T_NO_PV
+                return;
+#endif
                 const uint32_t v_lo = desc_lo_sw128(v_stage, kSlabBytes);
 #pragma unroll
-                for (int k = k0; k < k1; ++k)
+                for (int k = k0; k < k1; ++k) {
+#if defined(VPP_T_PV_KMAJOR)   // timing experiment: wrong results
+                    const uint32_t koff = ((k >> 2) * kSlabBytes + (k & 3) * 32) >> 4;
+                    mma_ts_lh(tO, tP + k * 8, desc_lo_sw128(v_stage, 16) + koff, kHi, kIdescQK, (!first || k > 0) ? 1u : 0u);
+#elif defined(VPP_T_PV_SS)     // timing experiment: wrong results
+                    const uint32_t koff = ((k >> 2) * kSlabBytes + (k & 3) * 32) >> 4;
+                    mma_ss_lh(tO, q_lo0 + koff, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
+#else
                     mma_ts_lh(tO, tP + k * 8, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
+#endif
+                }
             };
             while (true) {
                 const uint32_t slot = item_it & 1;
                 if (!wait1(bar_item_full + 8 * slot, (item_it >> 1) & 1, 301)) break;
                 const WorkUnit u = ring[slot].u;
                 const int valid = ring[slot].valid;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
+                mbar_arrive(bar_item_empty + 8 * slot);
                 ++item_it;
                 if (!valid) break;
                 const int n = u.kv_end - u.kv_begin;
@@ -276,6 +305,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_kv_full + 8 * stV, (kv_it / kWsStages) & 1, 304);
                     if (!ok) break;
                     ++kv_it;
+                    if (lane == 0) VPP_TR(0, jj, 0);
                     if (tile0 + kTileN > u.kv_len) {
                         ok = wait1(bar_vfix, vfix_it & 1, 305);
                         if (!ok) break;
@@ -287,6 +317,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_p_full, p_it & 1, 306);
                     if (!ok) break;
                     tc_fence_after();
+                    if (lane == 0) VPP_TR(0, jj, 1);
 #ifdef VPP_SPLIT_P
                     if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 4);
                     ok = wait1(bar_p_full_b, p_it & 1, 309);
@@ -296,14 +327,26 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #else
                     if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
 #endif
+                    if (lane == 0) VPP_TR(0, jj, 2);
                     if (has_next) {
+#ifdef VPP_TRACE
+                        if (lane == 0) {
+                            VPP_TR(0, jj, 8);
+                            const bool first_try = mbar_try_wait(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1);
+                            VPP_TR(0, jj, 9);
+                            if (blockIdx.x == 0 && item_it == 1 && jj >= 8 && jj < 40) g_trace[(jj - 8) * 64 + 10] = first_try;
+                        }
+#endif
                         ok = wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 307);
                         if (!ok) break;
+                        if (lane == 0) VPP_TR(0, jj, 7);
                         tc_fence_after();
+                        if (lane == 0) VPP_TR(0, jj, 3);
                         if (lane == 0) {
                             issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                             tc_commit(bar_s_full);
                         }
+                        if (lane == 0) VPP_TR(0, jj, 4);
                     } else if (lane == 0) {
                         tc_commit(bar_o_full);
                     }
@@ -311,6 +354,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_p_full + 8, p_it & 1, 308);
                     if (!ok) break;
                     tc_fence_after();
+                    if (lane == 0) VPP_TR(0, jj, 5);
 #ifdef VPP_SPLIT_P
                     if (lane == 0) issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 4);
                     ok = wait1(bar_p_full_b + 8, p_it & 1, 310);
@@ -333,12 +377,23 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             tc_commit(bar_o_full + 8);
                         }
                     }
+                    if (lane == 0) VPP_TR(0, jj, 6);
                     if (has_next) ++kv_it;
                     ++p_it;
                 }
                 if (!ok) break;
             }
         }
+#ifdef VPP_TRACE
+        else if (warp == 3 && lane == 0 && blockIdx.x == 0) {
+            // observer: when does each K/V stage of the first item really become full?
+            const uint32_t item_it = 1;
+            for (int i = 0; i < 2 * 40; ++i) {
+                if (!mbar_wait(bar_kv_full + 8 * (i % kWsStages), (i / kWsStages) & 1, s_abort, 999)) break;
+                VPP_TR(3, i >> 1, 6 + (i & 1));
+            }
+        }
+#endif
         // warps 2 and 3 have nothing to do until teardown
     } else {
         // ===================================== softmax groups =====================================
@@ -372,12 +427,14 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!ok) break;
                 ++s_it;
                 tc_fence_after();
+                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 0);
                 uint32_t s[128];
                 tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                 tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
                 tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(s[64]));
                 tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(s[96]));
                 tc_wait_ld();
+                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 1);
                 if (tile0 + kTileN - 1 > u.pos0) {  // diagonal tile: keys beyond the row's position are masked
                     const int lim = my_pos - tile0;  // columns <= lim are visible
 #pragma unroll
@@ -413,6 +470,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
                 const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 2);
                 float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -440,8 +498,10 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #endif
                 }
                 l_run += sum0 + sum1;
+                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 3);
                 tc_wait_st();
                 tc_fence_before();
+                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 4);
 #ifdef VPP_SPLIT_P
                 mbar_arrive(bar_pb);
 #else
