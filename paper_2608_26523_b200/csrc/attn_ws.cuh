@@ -32,6 +32,10 @@ constexpr int kWsStages = VPP_WS_STAGES;      // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 1024 /*barriers, ring*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
+#ifndef VPP_EMU_EVERY
+#define VPP_EMU_EVERY 0
+#endif
+constexpr int kEmuEvery = VPP_EMU_EVERY;      // 0: all exponentials on the SFU (measured fastest so far)
 
 #ifdef VPP_TRACE
 // Timing experiment only (never part of the product build): clock64 stamps of CTA 0's roles.
@@ -51,8 +55,6 @@ struct WsItem {
     int32_t pad[2];
 };
 
-__device__ __forceinline__ void setmaxnreg_dec56() { asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); }
-__device__ __forceinline__ void setmaxnreg_inc224() { asm volatile("setmaxnreg.inc.sync.aligned.u32 224;"); }
 
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -69,8 +71,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_q_full = sBar + 32;
     const uint32_t bar_q_empty = sBar + 40;
     const uint32_t bar_s_full = sBar + 48;       // [2]
-    const uint32_t bar_p_full = sBar + 64;       // [2 tiles] (first half of P)
-    const uint32_t bar_p_full_b = sBar + 104;    // [2 tiles] (second half of P)
+    const uint32_t bar_p_full = sBar + 64;       // [2]
     const uint32_t bar_o_full = sBar + 80;       // [2]
     const uint32_t bar_vfix = sBar + 96;
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
@@ -89,8 +90,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(bar_item_full + 8 * i, 1);
             mbar_init(bar_item_empty + 8 * i, 9);
             mbar_init(bar_s_full + 8 * i, 1);
-            mbar_init(bar_p_full + 8 * i, 128);
-            mbar_init(bar_p_full_b + 8 * i, 128);
+            mbar_init(bar_p_full + 8 * i, 4);   // one arrival per softmax warp
             mbar_init(bar_o_full + 8 * i, 1);
         }
         mbar_init(bar_q_full, 1);
@@ -121,7 +121,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int total_items = num_units * (p.num_q_heads / 2);
 
     if (warp < 4) {
-        setmaxnreg_dec56();
         if (warp == 0) {
             // ============================ scheduler + TMA producer ============================
             uint32_t item_it = 0, q_it = 0, kv_it = 0;
@@ -318,15 +317,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (!ok) break;
                     tc_fence_after();
                     if (lane == 0) VPP_TR(0, jj, 1);
-#ifdef VPP_SPLIT_P
-                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 4);
-                    ok = wait1(bar_p_full_b, p_it & 1, 309);
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 4, 8);
-#else
-                    if (lane == 0) issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
-#endif
+                    issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
                     if (lane == 0) VPP_TR(0, jj, 2);
                     if (has_next) {
 #ifdef VPP_TRACE
@@ -355,18 +346,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (!ok) break;
                     tc_fence_after();
                     if (lane == 0) VPP_TR(0, jj, 5);
-#ifdef VPP_SPLIT_P
-                    if (lane == 0) issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 4);
-                    ok = wait1(bar_p_full_b + 8, p_it & 1, 310);
-                    if (!ok) break;
-                    tc_fence_after();
-#endif
                     if (lane == 0) {
-#ifdef VPP_SPLIT_P
-                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 4, 8);
-#else
                         issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 8);
-#endif
                         tc_commit(bar_kv_empty + 8 * stV);
                         if (has_next) {
                             issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
@@ -397,14 +378,12 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // warps 2 and 3 have nothing to do until teardown
     } else {
         // ===================================== softmax groups =====================================
-        setmaxnreg_inc224();
         const int t = (warp - 4) >> 2;                 // query tile / softmax group
         const int row = ((warp & 3) << 5) | lane;      // row of the tile = TMEM lane
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tS = tmem_base + t * 128 + lane_off;
         const uint32_t tO = tmem_base + 256 + t * 128 + lane_off;
         const uint32_t bar_s = bar_s_full + 8 * t, bar_p = bar_p_full + 8 * t, bar_o = bar_o_full + 8 * t;
-        const uint32_t bar_pb = bar_p_full_b + 8 * t;
         uint32_t item_it = 0, s_it = 0, o_it = 0;
         const float sc = p.scale_log2e;
         while (true) {
@@ -429,25 +408,32 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_fence_after();
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 0);
                 uint32_t s[128];
+                const bool diag = tile0 + kTileN - 1 > u.pos0;  // keys beyond the row's position are masked
+                const int lim = my_pos - tile0;                 // columns <= lim are visible
+                float mx[8];
+                // the second half of the row is still in flight while the first half is reduced
                 tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                 tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
+                tc_wait_ld();
                 tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(s[64]));
                 tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(s[96]));
-                tc_wait_ld();
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 1);
-                if (tile0 + kTileN - 1 > u.pos0) {  // diagonal tile: keys beyond the row's position are masked
-                    const int lim = my_pos - tile0;  // columns <= lim are visible
 #pragma unroll
-                    for (int i = 0; i < 128; ++i)
-                        if (i > lim) s[i] = 0xff800000u;  // -inf
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (hh == 1) tc_wait_ld();
+                    if (diag) {
+#pragma unroll
+                        for (int i = 0; i < 64; ++i)
+                            if (hh * 64 + i > lim) s[hh * 64 + i] = 0xff800000u;  // -inf
+                    }
+#pragma unroll
+                    for (int i = 0; i < 64; i += 8)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float v = __uint_as_float(s[hh * 64 + i + k]);
+                            mx[k] = (hh == 0 && i == 0) ? v : fmaxf(mx[k], v);
+                        }
                 }
-                float mx[8];
-#pragma unroll
-                for (int k = 0; k < 8; ++k) mx[k] = __uint_as_float(s[k]);
-#pragma unroll
-                for (int i = 8; i < 128; i += 8)
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) mx[k] = fmaxf(mx[k], __uint_as_float(s[i + k]));
                 const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 const float m_new = fmaxf(mxa * sc, m_ref);
@@ -481,32 +467,25 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         const float p0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
                         const float p1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
 #else
-                        const float p0 = ex2(fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use));
-                        const float p1 = ex2(fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use));
+                        const float x0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
+                        const float x1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
+                        // optionally every kEmuEvery-th exponential runs on the FMA pipe instead of the SFU
+                        const float p0 = (kEmuEvery > 0 && (i % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x0) : ex2(x0);
+                        const float p1 = (kEmuEvery > 0 && ((i + 1) % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x1) : ex2(x1);
 #endif
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(tS + c * 16, pk);
-#ifdef VPP_SPLIT_P
-                    if (c == 1) {  // first 64 keys of P are in place: the MMA warp may start O += P V on them
-                        tc_wait_st();
-                        tc_fence_before();
-                        mbar_arrive(bar_p);
-                    }
-#endif
                 }
                 l_run += sum0 + sum1;
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 3);
                 tc_wait_st();
                 tc_fence_before();
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 4);
-#ifdef VPP_SPLIT_P
-                mbar_arrive(bar_pb);
-#else
-                mbar_arrive(bar_p);
-#endif
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_p);
             }
             if (!ok) break;
 

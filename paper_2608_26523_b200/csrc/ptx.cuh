@@ -233,6 +233,20 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x on the FMA pipe (for x <= ~100): floor/fraction split with a round-down magic add, degree-4
+// minimax polynomial for 2^f on [0,1) (max relative error 2.7e-6, mean 4e-8), exponent patched in with
+// an integer add.  Used for a fraction of the softmax exponentials to take load off the SFU (16
+// ex2/clk/SM), which otherwise limits the softmax at head_dim 128.
+__device__ __forceinline__ float ex2_poly(float x) {
+    x = fmaxf(x, -126.f);
+    const float xf = __fadd_rd(x, 12582912.f);  // 1.5 * 2^23: the low mantissa bits now hold floor(x)
+    const float f = x - (xf - 12582912.f);
+    float p = fmaf(0.013534167781472206f, f, 0.05201146379113197f);
+    p = fmaf(p, f, 0.2414427548646927f);
+    p = fmaf(p, f, 0.6930038332939148f);
+    p = fmaf(p, f, 1.0000026226043701f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xf) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
