@@ -153,6 +153,40 @@ vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t n
                          int32_t total_q, int32_t num_q_heads, int32_t head_dim_v, void *out,
                          float *lse, vpp_stream_t stream);
 
+/*
+ * Same operation as vpp_chunk_attn_fwd, for callers that cannot obtain device memory themselves.
+ * (The paper has no counterpart for this entry point: it is a packaging variant, not a method step.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin called inside a framework's
+ * captured or memory-planned region, a serving process whose device memory was handed out in full at
+ * start-up, a host thread that must not take the allocator's lock.  Such a caller still passes every
+ * input and output buffer; what it cannot supply is the workspace.  Here the workspace is a fixed
+ * array of VPP_STATIC_SCRATCH_BYTES inside the library, so `args->workspace` and
+ * `args->workspace_bytes` are ignored.
+ *
+ *  - The call allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ *  - Every device that loads the library holds the array (VPP_STATIC_SCRATCH_BYTES) until the
+ *    process exits.
+ *  - The first call on each device looks up the array's device address (a one-time set-up that is
+ *    not a stream operation); make that first call before starting any stream capture.
+ *  - A launch whose vpp_chunk_attn_workspace_size exceeds VPP_STATIC_SCRATCH_BYTES is refused
+ *    with VPP_ERR_WORKSPACE and nothing is enqueued; vpp_static_last_error() says how much was needed.
+ *    (Split-KV partials dominate: 4 * num_kv_splits * total_q * num_q_heads * (head_dim_v + 1) bytes.)
+ *  - All calls on a device share the one array, and it keeps whatever the previous call left there.
+ *    Nothing in it has to start at zero -- the work-decomposition kernel rewrites the header, the work
+ *    list and the per-row split counts of each launch before they are read -- but two calls that
+ *    overlap on the GPU (different streams, or graphs replayed concurrently) race on it.  Serialise them.
+ *  - Other errors and the meaning of *status are those of vpp_chunk_attn_fwd.
+ */
+#define VPP_STATIC_SCRATCH_BYTES (32u << 20)
+vpp_status vpp_chunk_attn_fwd_static(const vpp_chunk_attn_args *args, vpp_stream_t stream);
+
+/* Size of the built-in scratch array (VPP_STATIC_SCRATCH_BYTES of the library that was loaded). */
+size_t vpp_static_scratch_bytes(void);
+
+/* Thread-local detail of the last failure of vpp_chunk_attn_fwd_static on this host thread. */
+const char *vpp_static_last_error(void);
+
 /* Static description of a status code. */
 const char *vpp_status_string(vpp_status s);
 

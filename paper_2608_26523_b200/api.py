@@ -19,7 +19,8 @@ VPP_ERR_CUDA = -4
 VPP_ERR_TIMEOUT = -5
 
 EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_status_string",
-           "vpp_last_error", "vpp_last_launch_count"]
+           "vpp_last_error", "vpp_last_launch_count", "vpp_chunk_attn_fwd_static", "vpp_static_scratch_bytes",
+           "vpp_static_last_error"]
 
 
 class VppError(RuntimeError):
@@ -65,6 +66,10 @@ def load_library():
         lib.vpp_status_string.argtypes = [ctypes.c_int]
         lib.vpp_last_error.restype = ctypes.c_char_p
         lib.vpp_last_launch_count.restype = ctypes.c_int32
+        lib.vpp_chunk_attn_fwd_static.restype = ctypes.c_int
+        lib.vpp_chunk_attn_fwd_static.argtypes = [ctypes.POINTER(ChunkAttnArgs), ctypes.c_void_p]
+        lib.vpp_static_scratch_bytes.restype = ctypes.c_size_t
+        lib.vpp_static_last_error.restype = ctypes.c_char_p
         _lib = lib
     return _lib
 
@@ -122,6 +127,24 @@ def vpp_chunk_attn_fwd(args, stream=None):
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
     _check(load_library().vpp_chunk_attn_fwd(ctypes.byref(args), ctypes.c_void_p(stream)))
+
+
+def vpp_chunk_attn_fwd_static(args, stream=None):
+    """Same as vpp_chunk_attn_fwd but with the library's built-in scratch array as workspace.
+
+    For callers that cannot allocate device memory (the workspace fields of `args` are ignored).
+    Launches needing more than vpp_static_scratch_bytes() are refused; calls sharing a device must not
+    overlap on the GPU."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    lib = load_library()
+    rc = lib.vpp_chunk_attn_fwd_static(ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != VPP_OK:
+        raise VppError(rc, "%s: %s" % (lib.vpp_status_string(rc).decode(), lib.vpp_static_last_error().decode()))
+
+
+def vpp_static_scratch_bytes():
+    return int(load_library().vpp_static_scratch_bytes())
 
 
 def vpp_lse_merge(o_parts, lse_parts, out, lse=None, stream=None):
