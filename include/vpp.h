@@ -147,7 +147,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args *args, vpp_stream_t stre
  * lse_parts  fp32 [num_splits, total_q, num_q_heads]
  * out        bf16 [total_q, num_q_heads, head_dim_v]
  * lse        fp32 [total_q, num_q_heads] or NULL
- * head_dim_v must be a multiple of 8; pointers 16-byte aligned.
+ * head_dim_v must be a multiple of 8, num_splits at most 64; pointers 16-byte aligned.
  */
 vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t num_splits,
                          int32_t total_q, int32_t num_q_heads, int32_t head_dim_v, void *out,

@@ -346,7 +346,8 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     // ---- merge of split partials ----
     if (L.splits > 1) {
         const long long pairs = static_cast<long long>(a->total_q) * a->num_q_heads;
-        const long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+        long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+        if (blocks > 8ll * sms) blocks = 8ll * sms;
         vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
             ap.o_parts, ap.lse_parts, L.splits, a->total_q, a->num_q_heads, a->head_dim_v, row_splits,
             static_cast<__nv_bfloat16*>(a->out), a->lse);
@@ -363,13 +364,16 @@ vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t n
     if (num_splits <= 0 || total_q < 0 || num_q_heads <= 0 || head_dim_v <= 0)
         return fail(VPP_ERR_INVALID_ARG, "num_splits, num_q_heads, head_dim_v must be > 0 and total_q >= 0");
     if (head_dim_v % 8 != 0) return fail(VPP_ERR_UNSUPPORTED, "head_dim_v must be a multiple of 8");
+    if (num_splits > vpp::kMergeMaxSplits) return fail(VPP_ERR_UNSUPPORTED, "at most %d splits", vpp::kMergeMaxSplits);
     if (total_q == 0) return VPP_OK;
     if (!o_parts || !lse_parts || !out) return fail(VPP_ERR_INVALID_ARG, "o_parts, lse_parts and out must be non-null");
     if ((reinterpret_cast<uintptr_t>(o_parts) | reinterpret_cast<uintptr_t>(out)) & 15u)
         return fail(VPP_ERR_INVALID_ARG, "o_parts and out must be 16-byte aligned");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const long long pairs = static_cast<long long>(total_q) * num_q_heads;
-    const long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+    long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+    const long long cap = 8ll * sm_count_or_default();
+    if (blocks > cap) blocks = cap;
     vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
         o_parts, lse_parts, num_splits, total_q, num_q_heads, head_dim_v, nullptr, static_cast<__nv_bfloat16*>(out),
         lse);
