@@ -138,7 +138,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg4", "cfg5"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -149,6 +149,8 @@ def main():
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,
                        desc="cfg2: GQA Hq=64 Hkv=4 d=128, chunk 8192, 128-token pages, shuffled block_table"),
+          "cfg3": dict(prefixes=W.CFG3_PREFIXES, chunk=8192, hq=128, hkv=1,
+                       desc="cfg3: absorbed MLA Hq=128, one latent kv-head, Dqk=576 Dv=512, chunk 8192, 64-token pages"),
           "cfg4": dict(prefixes=W.CFG4_PREFIXES, chunk=16384, hq=64, hkv=8,
                        desc="cfg4: GQA Hq=64 Hkv=8 d=128, chunk 16384, 128-token pages, split-KV + merge"),
           "cfg5": dict(prefixes=[-1], chunk=16384, hq=64, hkv=8,
@@ -164,8 +166,9 @@ def main():
     config = {"workload": "%s, prefixes %s" % (WL["desc"], prefixes), "prefixes": prefixes, "chunk": chunk,
               "num_kv_splits": args.splits,
               "l2": "inputs larger than L2: each step cycles through %d MB of KV plus %d MB of Q per prefix point"
-              % (int((max(prefixes) + chunk) * WL["hkv"] * 128 * 2 * 2 / 1e6), int(chunk * WL["hq"] * 256 / 1e6))
-              if args.workload in ("cfg2", "cfg4") else
+              % (int((max(prefixes) + chunk) * (1152 if args.workload == "cfg3" else WL["hkv"] * 512) / 1e6),
+                 int(chunk * WL["hq"] * (1152 if args.workload == "cfg3" else 256) / 1e6))
+              if args.workload in ("cfg2", "cfg3", "cfg4") else
               ("whole problem is L2-resident: latency-bound case, no roofline claimed" if args.workload == "cfg1"
                else "inputs larger than L2 (about 3 GB of KV)")}
 
@@ -216,7 +219,8 @@ def main():
         for P in prefixes:
             runners.append(api.ChunkAttn(W.cfg1(P // 512, device=dev), num_kv_splits=args.splits))
     else:
-        base = (W.cfg2 if args.workload == "cfg2" else W.cfg4)(prefix=max_prefix, max_prefix=max_prefix, device=dev)
+        base = {"cfg2": W.cfg2, "cfg3": W.cfg3, "cfg4": W.cfg4}[args.workload](prefix=max_prefix, max_prefix=max_prefix,
+                                                                              device=dev)
         for P in prefixes:
             prob = base.with_chunk([P], [chunk], base.q)
             runners.append(api.ChunkAttn(prob, num_kv_splits=args.splits))
@@ -327,7 +331,7 @@ def main():
         curve.append({"prefix": P, "ms": round(ms, 4), "tflops": round(tf, 2), "frac_of_burst_peak": round(tf / burst, 4),
                       "frac_of_sustained_peak": round(tf / sustained, 4)})
     cost_curve = None
-    if len(prefixes) >= 3 and args.workload in ("cfg2", "cfg4"):
+    if len(prefixes) >= 3 and args.workload in ("cfg2", "cfg3", "cfg4"):
         # the paper's linear latency model (its Eq. 2) and balance identity (its Eq. 3) on the measured curve
         x = np.array(prefixes, dtype=np.float64); y = np.array(per_pt_ms, dtype=np.float64)
         b, a = np.polyfit(x, y, 1)

@@ -12,6 +12,7 @@
 
 #include "../../include/vpp.h"
 #include "attn_simple.cuh"
+#include "attn_mla.cuh"
 #include "attn_ws.cuh"
 #include "common.cuh"
 #include "merge.cuh"
@@ -180,7 +181,10 @@ bool force_simple() {
 bool use_ws_kernel(const vpp_chunk_attn_args* a) {
     return !force_simple() && ((a->num_q_heads / a->num_kv_heads) % 2 == 0);
 }
-int heads_per_item(const vpp_chunk_attn_args* a, Family) { return use_ws_kernel(a) ? 2 : 1; }
+int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
+    if (fam == Family::kMla576) return 1;
+    return use_ws_kernel(a) ? 2 : 1;
+}
 
 vpp::WorkspaceLayout layout_for(const vpp_chunk_attn_args* a, Family fam) {
     vpp::WorkspaceLayout L{};
@@ -242,7 +246,11 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         return fail(VPP_ERR_WORKSPACE, "workspace: need %zu bytes, got %zu", L.total, a->workspace_bytes);
     if (reinterpret_cast<uintptr_t>(a->workspace) & 255u)
         return fail(VPP_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
-    if (fam == Family::kMla576) return fail(VPP_ERR_UNSUPPORTED, "the (576, 512) kernel is not built yet");
+    if (fam == Family::kMla576 &&
+        (a->v_cache != a->k_cache || a->v_block_stride != a->k_block_stride || a->v_token_stride != a->k_token_stride ||
+         a->v_head_stride != a->k_head_stride))
+        return fail(VPP_ERR_UNSUPPORTED,
+                    "the (576, 512) kernel needs v_cache to alias k_cache with the same strides (V = first 512 features)");
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     g_launches = 0;
@@ -256,7 +264,8 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     const bool paged = a->block_table != nullptr;
     const int B = paged ? a->block_size : a->max_seq_len;
     const int n_blocks = paged ? a->num_blocks : a->num_reqs;
-    const int box_rows = paged ? (B < vpp::kTileN ? B : vpp::kTileN) : vpp::kTileN;
+    const int tile_n = fam == Family::kMla576 ? vpp::kMlaTileN : vpp::kTileN;  // keys per KV tile of the kernel
+    const int box_rows = paged ? (B < tile_n ? B : tile_n) : tile_n;
 
     // ---- tensor maps ----
     CUtensorMap tm_q, tm_k, tm_v;
@@ -276,7 +285,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         const uint32_t b[4] = {64, static_cast<uint32_t>(box_rows), 1, 1};
         if (!make_tmap(&tm_k, a->k_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k) failed");
     }
-    {
+    if (fam != Family::kMla576) {
         const uint64_t d[4] = {static_cast<uint64_t>(a->head_dim_v), static_cast<uint64_t>(B),
                                static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
         const uint64_t s[3] = {static_cast<uint64_t>(a->v_token_stride) * 2, static_cast<uint64_t>(a->v_head_stride) * 2,
@@ -331,7 +340,11 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
 
     const int sms = sm_count_or_default();
     cudaError_t ce;
-    if (use_ws_kernel(a)) {
+    if (fam == Family::kMla576) {
+        auto kern = vpp::attn_mla_kernel;
+        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, ap, box_rows);
+    } else if (use_ws_kernel(a)) {
         auto kern = vpp::attn128_ws_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
         if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);

@@ -33,6 +33,11 @@ def test_cfg4_million_token_split_kv(prefix, splits):
                   num_kv_splits=splits, n_random=128)
 
 
+@pytest.mark.parametrize("prefix", [0, 65536, 516096])
+def test_cfg3_absorbed_mla(prefix):
+    check_sampled(W.cfg3(prefix=prefix, device="cuda"), "cfg3 P=%d" % prefix, n_random=96)
+
+
 def test_cfg5_mixed_varlen_batch():
     prob = W.cfg5(device="cuda")
     assert prob.total_q == 16384 and prob.num_reqs == 32

@@ -51,6 +51,38 @@ def test_adversarial_shapes(case, splits):
     print(s)
 
 
+MLA_CASES = [
+    # prefix_lens, chunk_lens, hq, block_size      (absorbed MLA: Dqk 576, Dv 512, one shared latent kv-head)
+    ([0], [1], 2, None),
+    ([0], [129], 4, 64),
+    ([63], [2], 2, 64),
+    ([300], [77], 4, 16),
+    ([1000, 0, 17, 511], [200, 0, 300, 129], 8, 32),
+    ([4095], [257], 4, 256),
+    ([513], [640], 4, None),
+]
+
+
+@pytest.mark.parametrize("case", range(len(MLA_CASES)))
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_mla_adversarial_shapes(case, splits):
+    P, C, hq, bs = MLA_CASES[case]
+    prob = W.make_problem(2000 + case, P, C, hq, 1, 576, 512, block_size=bs, std=0.5, scale=1.0 / 192 ** 0.5,
+                          v_aliases_k=True)
+    s, _ = full_check(prob, num_kv_splits=splits, label="mla case %d S=%d" % (case, splits))
+    print(s)
+
+
+def test_mla_requires_aliased_values():
+    prob = W.make_problem(2100, [10], [20], 2, 1, 576, 512, block_size=16, std=0.5, v_aliases_k=True).to("cuda")
+    runner = api.ChunkAttn(prob)
+    other = torch.zeros_like(prob.k_cache)
+    runner.args.v_cache = other.data_ptr()
+    with pytest.raises(api.VppError) as ei:
+        runner.run()
+    assert ei.value.status == api.VPP_ERR_UNSUPPORTED
+
+
 def test_outputs_outside_the_launch_are_untouched():
     """Canary rows around out / lse keep their value."""
     prob = W.make_problem(77, [40], [100], 4, 2, 128, 128, block_size=64).to("cuda")
