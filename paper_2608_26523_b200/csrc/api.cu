@@ -294,6 +294,20 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_v, a->v_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(v) failed");
     }
 
+    CUtensorMap tm_k4, tm_k5;
+    if (fam == Family::kMla576) {
+        // rank-5 views (64 columns, keys, slab, head, block): boxes of 4 / 5 slabs x 64 keys
+        const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
+                               static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
+        const uint64_t s[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
+                               static_cast<uint64_t>(a->k_block_stride) * 2};
+        const uint32_t rows = static_cast<uint32_t>(box_rows);
+        const uint32_t b4[5] = {64, rows, 4, 1, 1};
+        const uint32_t b5[5] = {64, rows, 5, 1, 1};
+        if (!make_tmap(&tm_k4, a->k_cache, 5, d, s, b4) || !make_tmap(&tm_k5, a->k_cache, 5, d, s, b5))
+            return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k slab groups) failed");
+    }
+
     // ---- work decomposition ----
     int32_t* row_splits = reinterpret_cast<int32_t*>(ws + L.row_splits);
     vpp::PrepParams pp{};
@@ -343,7 +357,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, ap, box_rows);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, tm_k4, tm_k5, ap, box_rows);
     } else if (use_ws_kernel(a)) {
         auto kern = vpp::attn128_ws_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);

@@ -49,8 +49,12 @@ __device__ __forceinline__ int mla_slab_order(int pass, int i) {
 }
 
 __global__ void __launch_bounds__(kMlaThreads, 1)
-attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, const AttnParams p,
+attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_k4, const __grid_constant__ CUtensorMap tm_k5, const AttnParams p,
                 const int kv_box_rows) {
+    // tm_k loads one 64-column slab of kv_box_rows keys; tm_k4 / tm_k5 are rank-5 views of the same cache
+    // (64 columns, keys, slab index, head, block) whose boxes cover 4 / 5 consecutive slabs of 64 keys, so
+    // that a whole slab group arrives with one copy instruction (used when a KV tile lies in one page).
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -65,8 +69,10 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const uint32_t bar_p_full = sBar + 64;       // [2]
     const uint32_t bar_o_full = sBar + 80;
     const uint32_t bar_vfix = sBar + 88;
-    const uint32_t bar_k_full = sBar + 128;      // [9]
-    const uint32_t bar_k_empty = sBar + 256;     // [9]
+    // The nine K slabs of a tile travel as two groups: group 0 = the five slabs that are not values of the
+    // current pass, group 1 = its four value slabs.
+    const uint32_t bar_k_full = sBar + 128;      // [2 groups]
+    const uint32_t bar_k_empty = sBar + 144;     // [2 groups]
     uint8_t* gen_bar = gen_base + kMlaSlabs * (kMlaQSlab + kMlaKSlab);
     volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 512);
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 516);
@@ -87,7 +93,7 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(bar_q_empty, 1);
         mbar_init(bar_o_full, 1);
         mbar_init(bar_vfix, 1);
-        for (int i = 0; i < kMlaSlabs; ++i) {
+        for (int i = 0; i < 2; ++i) {
             mbar_init(bar_k_full + 8 * i, 1);
             mbar_init(bar_k_empty + 8 * i, 1);
         }
@@ -95,6 +101,8 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         *s_abort = 0;
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
+        prefetch_tmap(&tm_k4);
+        prefetch_tmap(&tm_k5);
     }
     __syncthreads();
     if (warp == 0) {
@@ -165,28 +173,55 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int j = t_lo; j < t_hi && ok; ++j) {
                     const int tile0 = j * kMlaTileN;
                     if (lane == 0) {
-                        for (int i = 0; i < kMlaSlabs && ok; ++i) {
-                            const int s = mla_slab_order(pass, i);
-                            ok = mbar_wait(bar_k_empty + 8 * s, (fill & 1) ^ 1, s_abort, 503);
-                            if (!ok) break;
-                            const uint32_t full = bar_k_full + 8 * s;
-                            mbar_arrive_expect_tx(full, kMlaKSlab);
-                            for (int off = 0; off < kMlaTileN; off += kv_box_rows) {
-                                const int pos = tile0 + off;
-                                int blk, slot_in;
-                                if (p.block_table == nullptr) {
-                                    blk = u.req;
-                                    slot_in = pos;
-                                } else if (pos < u.kv_len) {
-                                    blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                        // page lookup once per tile (not per slab): a dependent global load costs more than a slab's MMAs
+                        int blk[4], slot_in[4];
+                        int np = 0;
+                        for (int off = 0; off < kMlaTileN; off += kv_box_rows, ++np) {
+                            const int pos = tile0 + off;
+                            if (p.block_table == nullptr) {
+                                blk[np] = u.req;
+                                slot_in[np] = pos;
+                            } else if (pos < u.kv_len) {
+                                blk[np] = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
                                                 (pos >> p.block_shift));
-                                    slot_in = pos & ((1 << p.block_shift) - 1);
-                                } else {
-                                    blk = p.num_blocks;  // out of range: the copy engine fills zeros
-                                    slot_in = 0;
-                                }
-                                tma_load_4d(sK + s * kMlaKSlab + off * 128, &tm_k, full, 64 * s, slot_in, 0, blk);
+                                slot_in[np] = pos & ((1 << p.block_shift) - 1);
+                            } else {
+                                blk[np] = p.num_blocks;  // out of range: the copy engine fills zeros
+                                slot_in[np] = 0;
                             }
+                        }
+                        if (j == t_lo) {
+                            // the physical slabs change groups between passes: both groups of the previous tile
+                            // must have been released before anything of this pass is loaded
+                            ok = mbar_wait(bar_k_empty + 8, (fill & 1) ^ 1, s_abort, 505);
+                        }
+                        for (int grp = 0; grp < 2 && ok; ++grp) {
+                            VPP_TR(3, j - t_lo, grp * 3 + 0);
+                            ok = mbar_wait(bar_k_empty + 8 * grp, (fill & 1) ^ 1, s_abort, 503);
+                            if (!ok) break;
+                            VPP_TR(3, j - t_lo, grp * 3 + 1);
+                            const uint32_t full = bar_k_full + 8 * grp;
+                            const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
+                            mbar_arrive_expect_tx(full, (i1 - i0) * kMlaKSlab);
+                            if (kv_box_rows == kMlaTileN) {
+                                // one page per tile: whole runs of consecutive slabs per instruction
+                                if (grp == 1) {
+                                    tma_load_5d(sK + pass * 4 * kMlaKSlab, &tm_k4, full, 0, slot_in[0], pass * 4, 0, blk[0]);
+                                } else if (pass == 0) {
+                                    tma_load_5d(sK + 4 * kMlaKSlab, &tm_k5, full, 0, slot_in[0], 4, 0, blk[0]);
+                                } else {
+                                    tma_load_5d(sK, &tm_k4, full, 0, slot_in[0], 0, 0, blk[0]);
+                                    tma_load_4d(sK + 8 * kMlaKSlab, &tm_k, full, 64 * 8, slot_in[0], 0, blk[0]);
+                                }
+                            } else {
+                                for (int i = i0; i < i1; ++i) {
+                                    const int s = mla_slab_order(pass, i);
+                                    for (int q = 0; q < np; ++q)
+                                        tma_load_4d(sK + s * kMlaKSlab + q * kv_box_rows * 128, &tm_k, full, 64 * s,
+                                                    slot_in[q], 0, blk[q]);
+                                }
+                            }
+                            VPP_TR(3, j - t_lo, grp * 3 + 2);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -194,10 +229,8 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (tile0 + kMlaTileN > u.kv_len) {
                         // keys at or beyond kv_len do not exist: zero their rows in the four value slabs of this
                         // pass so that 0 * garbage cannot poison O; the MMA thread waits for bar_vfix on such a tile
-                        for (int i = 0; i < 4 && ok; ++i) {
-                            if (lane == 0) ok = mbar_wait(bar_k_full + 8 * (pass * 4 + i), fill & 1, s_abort, 504);
-                            ok = __shfl_sync(0xffffffffu, ok, 0);
-                        }
+                        if (lane == 0) ok = mbar_wait(bar_k_full + 8, fill & 1, s_abort, 504);
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
                         if (!ok) break;
                         const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
                         const uint4 z = make_uint4(0, 0, 0, 0);
@@ -228,11 +261,12 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t v_lo = desc_lo_sw128(sK, kMlaKSlab);
         uint32_t item_it = 0, q_it = 0, fill = 0, tc = 0, vfix_it = 0;
         // score MMAs of KV tile number `fl` (global count) for slabs order[i0..i1) of `pass`
-        auto issue_qk = [&](uint32_t tS, int pass, int i0, int i1, uint32_t fl) -> bool {
+        auto issue_qk = [&](uint32_t tS, int pass, int grp, uint32_t fl) -> bool {
+            if (!mbar_wait(bar_k_full + 8 * grp, fl & 1, s_abort, 601)) return false;
+            tc_fence_after();
+            const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
             for (int i = i0; i < i1; ++i) {
                 const int s = mla_slab_order(pass, i);
-                if (!mbar_wait(bar_k_full + 8 * s, fl & 1, s_abort, 601)) return false;
-                tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     mma_ss_lh(tS, q_lo + ((s * kMlaQSlab + kk * 32) >> 4), k_lo + ((s * kMlaKSlab + kk * 32) >> 4), kHi,
@@ -255,11 +289,11 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ++q_it;
             bool ok = true;
             for (int pass = 0; pass < 2 && ok; ++pass) {
-                // first tile of the pass: all nine slabs
-                ok = issue_qk(tmem_base + (tc & 1) * 64, pass, 0, 5, fill);
+                // first tile of the pass: both groups
+                ok = issue_qk(tmem_base + (tc & 1) * 64, pass, 0, fill);
                 if (!ok) break;
-                for (int i = 0; i < 5; ++i) tc_commit(bar_k_empty + 8 * mla_slab_order(pass, i));
-                ok = issue_qk(tmem_base + (tc & 1) * 64, pass, 5, 9, fill);
+                tc_commit(bar_k_empty);
+                ok = issue_qk(tmem_base + (tc & 1) * 64, pass, 1, fill);
                 if (!ok) break;
                 tc_commit(bar_s_full + 8 * (tc & 1));
                 if (n == 1 && pass == 1) tc_commit(bar_q_empty);
@@ -268,31 +302,47 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t b = tc & 1;               // score buffer of tile jj
                     const uint32_t tS = tmem_base + b * 64;
                     const bool has_next = jj + 1 < n;
-                    if (has_next) {
-                        // non-value slabs of the next tile: overlaps the softmax of this one
-                        ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 0, 5, fill + 1);
+                    bool early = false;
+                    VPP_TR(0, jj, 0);
+                    if (has_next && mbar_try_wait(bar_k_full, (fill + 1) & 1)) {
+                        // the non-value slabs of the next tile are already here: their score MMAs overlap the
+                        // softmax of this tile (if they are not, P V of this tile must not wait for them)
+                        ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 0, fill + 1);
                         if (!ok) break;
-                        for (int i = 0; i < 5; ++i) tc_commit(bar_k_empty + 8 * mla_slab_order(pass, i));
+                        tc_commit(bar_k_empty);
+                        early = true;
                     }
                     if (tile0 + kMlaTileN > u.kv_len) {
                         ok = mbar_wait(bar_vfix, vfix_it & 1, s_abort, 604);
                         if (!ok) break;
                         ++vfix_it;
                     }
+                    VPP_TR(0, jj, 1);
                     ok = mbar_wait(bar_p_full + 8 * b, (tc >> 1) & 1, s_abort, 605);
                     if (!ok) break;
                     tc_fence_after();
+                    VPP_TR(0, jj, 2);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         mma_ts_lh(tO, tS + kk * 8, v_lo + ((pass * 4 * kMlaKSlab + kk * 2048) >> 4), kHi, kIdescPV,
                                   (jj > 0 || kk > 0) ? 1u : 0u);
-                    for (int i = 0; i < 4; ++i) tc_commit(bar_k_empty + 8 * (pass * 4 + i));
+                    tc_commit(bar_k_empty + 8);
+                    VPP_TR(0, jj, 3);
                     ++fill;
                     ++tc;
                     if (has_next) {
-                        ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 5, 9, fill);
+                        if (!early) {
+                            ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 0, fill);
+                            if (!ok) break;
+                            tc_commit(bar_k_empty);
+                        }
+                        VPP_TR(0, jj, 4);
+                        if (!mbar_wait(bar_k_full + 8, fill & 1, s_abort, 606)) { ok = false; break; }
+                        VPP_TR(0, jj, 5);
+                        ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 1, fill);
                         if (!ok) break;
                         tc_commit(bar_s_full + 8 * (b ^ 1));
+                        VPP_TR(0, jj, 6);
                         if (jj + 2 == n && pass == 1) tc_commit(bar_q_empty);
                     } else {
                         tc_commit(bar_o_full);
@@ -332,6 +382,7 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!ok) break;
                     ++tc;
                     tc_fence_after();
+                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 0);
                     uint32_t s[64];
                     tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                     tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
@@ -370,6 +421,7 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 1);
                     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
@@ -387,6 +439,7 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     l_run += sum0 + sum1;
                     tc_wait_st();
                     tc_fence_before();
+                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 2);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_p_full + 8 * b);
                 }

@@ -37,17 +37,6 @@ constexpr float kRescaleThreshold = 8.f;      // log2 units
 #endif
 constexpr int kEmuEvery = VPP_EMU_EVERY;      // 0: all exponentials on the SFU (measured fastest so far)
 
-#ifdef VPP_TRACE
-// Timing experiment only (never part of the product build): clock64 stamps of CTA 0's roles.
-__device__ long long g_trace[64 * 32];
-#define VPP_TR(role, jj, k)                                                                     \
-    do {                                                                                        \
-        if (blockIdx.x == 0 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
-    } while (0)
-#else
-#define VPP_TR(role, jj, k) do {} while (0)
-#endif
-
 struct WsItem {
     WorkUnit u;
     int32_t h0;     // first of the two q-heads
