@@ -294,6 +294,24 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_v, a->v_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(v) failed");
     }
 
+    CUtensorMap tm_q2, tm_k2, tm_v2;
+    if (fam == Family::kGqa128) {
+        // the 128 features viewed as (64, 2): a box holds both 64-column slabs of a tile
+        const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), 2, static_cast<uint64_t>(a->num_q_heads)};
+        const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
+                                static_cast<uint64_t>(a->head_dim_qk) * 2};
+        const uint32_t bq[4] = {64, static_cast<uint32_t>(vpp::kTileM), 2, 1};
+        if (!make_tmap(&tm_q2, a->q, 4, dq, sq, bq)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(q tiles) failed");
+        const uint64_t d[5] = {64, static_cast<uint64_t>(B), 2, static_cast<uint64_t>(a->num_kv_heads),
+                               static_cast<uint64_t>(n_blocks)};
+        const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
+                                static_cast<uint64_t>(a->k_block_stride) * 2};
+        const uint64_t sv[4] = {static_cast<uint64_t>(a->v_token_stride) * 2, 128, static_cast<uint64_t>(a->v_head_stride) * 2,
+                                static_cast<uint64_t>(a->v_block_stride) * 2};
+        const uint32_t b5[5] = {64, static_cast<uint32_t>(box_rows), 2, 1, 1};
+        if (!make_tmap(&tm_k2, a->k_cache, 5, d, sk, b5) || !make_tmap(&tm_v2, a->v_cache, 5, d, sv, b5))
+            return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
+    }
     CUtensorMap tm_k4, tm_k5;
     if (fam == Family::kMla576) {
         // rank-5 views (64 columns, keys, slab, head, block): boxes of 4 / 5 slabs x 64 keys
@@ -361,7 +379,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     } else if (use_ws_kernel(a)) {
         auto kern = vpp::attn128_ws_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, ap, box_rows);
     } else {
         auto kern = vpp::attn128_simple_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);

@@ -47,7 +47,13 @@ struct WsItem {
 
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p, const int kv_box_rows) {
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_q2,
+                  const __grid_constant__ CUtensorMap tm_k2, const __grid_constant__ CUtensorMap tm_v2,
+                  const AttnParams p, const int kv_box_rows) {
+    // tm_q2 / tm_k2 / tm_v2 are views of the same tensors with the 128 features split into (64, 2): one box
+    // of them brings both 64-column slabs of a 128-row tile, i.e. a whole tile per copy instruction.  Issuing a
+    // copy costs the producer thread several hundred cycles, so fewer, larger copies matter.  tm_k / tm_v
+    // (one slab of kv_box_rows keys per box) serve pages smaller than a KV tile.
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -94,6 +100,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
+        prefetch_tmap(&tm_q2);
+        prefetch_tmap(&tm_k2);
+        prefetch_tmap(&tm_v2);
     }
     __syncthreads();
     if (warp == 2) {
@@ -145,10 +154,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 202);
                     if (ok) {
                         mbar_arrive_expect_tx(bar_q_full, 2 * kTileBytes);
-                        tma_load_3d(sQ, &tm_q, bar_q_full, 0, h0, u.q_row0);
-                        tma_load_3d(sQ + kSlabBytes, &tm_q, bar_q_full, 64, h0, u.q_row0);
-                        tma_load_3d(sQ + kTileBytes, &tm_q, bar_q_full, 0, h0 + 1, u.q_row0);
-                        tma_load_3d(sQ + kTileBytes + kSlabBytes, &tm_q, bar_q_full, 64, h0 + 1, u.q_row0);
+                        tma_load_4d(sQ, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0);
+                        tma_load_4d(sQ + kTileBytes, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0 + 1);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -170,6 +177,22 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             if (ok) {
                                 mbar_arrive_expect_tx(full, kTileBytes);
                                 const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+                                const CUtensorMap* tm2 = which == 0 ? &tm_k2 : &tm_v2;
+                                if (kv_box_rows == kTileN) {
+                                    int blk, slot_in;
+                                    if (p.block_table == nullptr) {
+                                        blk = u.req;
+                                        slot_in = tile0;
+                                    } else if (tile0 < u.kv_len) {
+                                        blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                                    (tile0 >> p.block_shift));
+                                        slot_in = tile0 & ((1 << p.block_shift) - 1);
+                                    } else {
+                                        blk = p.num_blocks;
+                                        slot_in = 0;
+                                    }
+                                    tma_load_5d(dst, tm2, full, 0, slot_in, 0, g, blk);
+                                } else
                                 for (int off = 0; off < kTileN; off += kv_box_rows) {
                                     const int pos = tile0 + off;
                                     int blk, slot_in;
