@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-from paper_2608_26523_b200 import workloads as W
+from paper_2608_26523_b200 import dist as D, workloads as W
 
 METRIC = "chunk-attn TFLOP/s and % dense BF16 peak vs prefix length (1 B200)"
 UNIT = "TFLOP/s"
@@ -207,7 +207,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+        D.init("nccl", dev)
     api.load_library()
 
     max_prefix = max(prefixes)
@@ -237,10 +237,7 @@ def main():
                 events[i][1].record(stream)
 
     def barrier():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        D.barrier(dev)
 
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
@@ -312,11 +309,10 @@ def main():
 
     # ---- max over ranks ----
     if world > 1:
-        t = torch.tensor([total_ms, e2e[1] if e2e else 0.0], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t[0])
+        t = D.max_over_ranks([total_ms, e2e[1] if e2e else 0.0], dev)
+        total_ms = t[0]
         if e2e:
-            e2e = (e2e[0], float(t[1]), e2e[2], e2e[3], e2e[4])
+            e2e = (e2e[0], t[1], e2e[2], e2e[3], e2e[4])
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

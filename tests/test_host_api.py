@@ -1,0 +1,143 @@
+"""Host-side behaviour of the C ABI that needs no GPU: the library loads, exports every symbol that
+include/vpp.h declares, sizes workspaces, and rejects bad arguments before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2608_26523_b200 import api, workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2608_26523_b200 import build
+    build.build()                      # nvcc cross-compiles without a GPU
+    return api.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "vpp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vpp_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert {"vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_chunk_attn_workspace_size",
+            "vpp_chunk_attn_fwd_static"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(api.EXPORTS) == set(names)
+
+
+def test_status_strings(lib):
+    for code in (0, -1, -2, -3, -4, -5):
+        assert lib.vpp_status_string(code).decode() != "unknown status"
+    assert lib.vpp_status_string(-99).decode() == "unknown status"
+
+
+def small_args(**kw):
+    p = W.make_problem(5, [10], [20], kw.pop("hq", 4), kw.pop("hkv", 2), kw.pop("dqk", 128), kw.pop("dv", 128),
+                       block_size=kw.pop("block_size", 16), v_aliases_k=kw.pop("alias", False))
+    a = api.make_args(p.q, p.k_cache, p.v_cache, p.block_table, p.prefix_len, p.chunk_len, p.block_size,
+                      p.max_seq_len, p.scale, **kw)
+    a._keep = p
+    return a
+
+
+def test_workspace_size_grows_with_splits(lib):
+    base = api.vpp_chunk_attn_workspace_size(small_args(num_kv_splits=1))
+    split = api.vpp_chunk_attn_workspace_size(small_args(num_kv_splits=4))
+    assert 0 < base < split
+    # partials: S * T * Hq * (Dv + 1) floats
+    assert split - base >= 4 * 20 * 4 * 129 * 4
+
+
+def test_layout_of_args_struct_matches_header(tmp_path):
+    """The ctypes mirror has the size and field offsets a C compiler gives the header's struct."""
+    import subprocess
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "vpp.h"\n'
+                   'int main(void){printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(vpp_chunk_attn_args),'
+                   'offsetof(vpp_chunk_attn_args, block_table), offsetof(vpp_chunk_attn_args, num_reqs),'
+                   'offsetof(vpp_chunk_attn_args, softmax_scale), offsetof(vpp_chunk_attn_args, out),'
+                   'offsetof(vpp_chunk_attn_args, status));return 0;}\n')
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    c = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    A = api.ChunkAttnArgs
+    assert c == [ctypes.sizeof(A), A.block_table.offset, A.num_reqs.offset, A.softmax_scale.offset, A.out.offset,
+                 A.status.offset]
+
+
+@pytest.mark.parametrize("mutate,status", [
+    (lambda a: setattr(a, "head_dim_qk", 96), api.VPP_ERR_UNSUPPORTED),
+    (lambda a: setattr(a, "num_kv_heads", 3), api.VPP_ERR_INVALID_ARG),
+    (lambda a: setattr(a, "softmax_scale", 0.0), api.VPP_ERR_INVALID_ARG),
+    (lambda a: setattr(a, "num_kv_splits", 65), api.VPP_ERR_INVALID_ARG),
+    (lambda a: setattr(a, "block_size", 24), api.VPP_ERR_UNSUPPORTED),
+    (lambda a: setattr(a, "k_token_stride", 100), api.VPP_ERR_INVALID_ARG),
+    (lambda a: setattr(a, "q", None), api.VPP_ERR_INVALID_ARG),
+    (lambda a: setattr(a, "q", a.q + 2), api.VPP_ERR_INVALID_ARG),          # misaligned
+    (lambda a: setattr(a, "workspace_bytes", 16), api.VPP_ERR_WORKSPACE),
+])
+def test_bad_arguments_are_rejected_before_any_launch(lib, mutate, status):
+    a = small_args()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8)
+    out = torch.zeros(20, 4, 128, dtype=torch.bfloat16)
+    a.workspace, a.workspace_bytes, a.out = ws.data_ptr() + (-ws.data_ptr() % 256), 1 << 19, out.data_ptr()
+    mutate(a)
+    with pytest.raises(api.VppError) as ei:
+        api.vpp_chunk_attn_fwd(a, stream=0)
+    assert ei.value.status == status
+    assert str(ei.value)
+
+
+def test_mla_shape_needs_aliased_values(lib):
+    a = small_args(hq=4, hkv=1, dqk=576, dv=512, alias=True)
+    ws = torch.zeros(1 << 22, dtype=torch.uint8)
+    out = torch.zeros(20, 4, 512, dtype=torch.bfloat16)
+    a.workspace, a.workspace_bytes, a.out = ws.data_ptr() + (-ws.data_ptr() % 256), 1 << 21, out.data_ptr()
+    a.v_cache = a.v_cache + 1152
+    with pytest.raises(api.VppError) as ei:
+        api.vpp_chunk_attn_fwd(a, stream=0)
+    assert ei.value.status == api.VPP_ERR_UNSUPPORTED
+
+
+def test_merge_argument_checks(lib):
+    with pytest.raises(api.VppError) as ei:
+        _check = lib.vpp_lse_merge(None, None, 0, 4, 4, 128, None, None, None)
+        api._check(_check)
+    assert ei.value.status == api.VPP_ERR_INVALID_ARG
+    rc = lib.vpp_lse_merge(None, None, 65, 4, 4, 128, None, None, None)
+    assert rc == api.VPP_ERR_UNSUPPORTED
+    assert lib.vpp_lse_merge(None, None, 2, 0, 4, 128, None, None, None) == api.VPP_OK     # nothing to do
+
+
+def test_static_entry_point_refuses_oversized_launch_on_host(lib):
+    p = W.make_problem(6, [0], [4096], 8, 2, 128, 128, block_size=128)
+    a = api.make_args(p.q, p.k_cache, p.v_cache, p.block_table, p.prefix_len, p.chunk_len, p.block_size,
+                      p.max_seq_len, p.scale, num_kv_splits=16)
+    assert api.vpp_chunk_attn_workspace_size(a) > api.vpp_static_scratch_bytes()
+    with pytest.raises(api.VppError) as ei:
+        api.vpp_chunk_attn_fwd_static(a, stream=0)
+    assert ei.value.status == api.VPP_ERR_WORKSPACE
+
+
+def test_cfg5_lengths_recipe():
+    L, C, P = W.cfg5_lengths()
+    assert len(L) == 32 and sum(C) == 16384
+    assert all(1024 <= l <= 262144 for l in L)
+    assert all(64 <= c <= min(l, 2048) for c, l in zip(C, L))
+    assert all(0 <= p <= l - c for p, c, l in zip(P, C, L))
+    assert W.cfg5_lengths() == (L, C, P)            # seeded
+
+
+def test_flop_count_is_the_exact_causal_count():
+    p = W.make_problem(7, [5, 0], [3, 2], 4, 2, 16, 8, block_size=None)
+    pairs = (3 * 5 + 3 * 4 // 2) + (2 * 0 + 2 * 3 // 2)
+    assert p.pairs() == pairs and p.flops() == 2 * 4 * (16 + 8) * pairs
