@@ -13,6 +13,7 @@
 #include "../../include/vpp.h"
 #include "attn_simple.cuh"
 #include "attn_mla.cuh"
+#include "attn_mla2.cuh"
 #include "attn_ws.cuh"
 #include "common.cuh"
 #include "merge.cuh"
@@ -181,6 +182,15 @@ bool force_simple() {
 bool use_ws_kernel(const vpp_chunk_attn_args* a) {
     return !force_simple() && ((a->num_q_heads / a->num_kv_heads) % 2 == 0);
 }
+// The pair-of-SMs MLA kernel needs every 64-key group of a KV tile inside one page; smaller pages take the
+// single-CTA two-pass kernel.  VPP_MLA_SINGLE=1 forces the latter (debugging aid, read once).
+bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
+    static const bool force_single = [] {
+        const char* e = std::getenv("VPP_MLA_SINGLE");
+        return e && e[0] == '1';
+    }();
+    return !force_single && (a->block_table == nullptr || a->block_size >= 64) && sm_count_or_default() >= 2;
+}
 int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     if (fam == Family::kMla576) return 1;
     return use_ws_kernel(a) ? 2 : 1;
@@ -312,6 +322,24 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_k2, a->k_cache, 5, d, sk, b5) || !make_tmap(&tm_v2, a->v_cache, 5, d, sv, b5))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
     }
+    CUtensorMap tm_q9, tm_k9, tm_v2m;
+    const bool mla_pair = fam == Family::kMla576 && use_mla_pair_kernel(a);
+    if (mla_pair) {
+        const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), static_cast<uint64_t>(vpp::kMlaSlabs),
+                                static_cast<uint64_t>(a->num_q_heads)};
+        const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
+                                static_cast<uint64_t>(a->head_dim_qk) * 2};
+        const uint32_t bq[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};
+        const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
+                               static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
+        const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
+                                static_cast<uint64_t>(a->k_block_stride) * 2};
+        const uint32_t b9[5] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1, 1};
+        const uint32_t b2[5] = {64, 64, 2, 1, 1};
+        if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) || !make_tmap(&tm_k9, a->k_cache, 5, d, sk, b9) ||
+            !make_tmap(&tm_v2m, a->k_cache, 5, d, sk, b2))
+            return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");
+    }
     CUtensorMap tm_k4, tm_k5;
     if (fam == Family::kMla576) {
         // rank-5 views (64 columns, keys, slab, head, block): boxes of 4 / 5 slabs x 64 keys
@@ -372,7 +400,11 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
 
     const int sms = sm_count_or_default();
     cudaError_t ce;
-    if (fam == Family::kMla576) {
+    if (mla_pair) {
+        auto kern = vpp::attn_mla2_kernel;
+        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
+        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, tm_v2m, ap);
+    } else if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
         if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, tm_k4, tm_k5, ap, box_rows);

@@ -1,0 +1,585 @@
+// Chunked-prefill attention for absorbed MLA (576-wide keys, values = first 512 features of the same row)
+// on a pair of SMs: a 2-CTA cluster issues tcgen05.mma with cta_group::2.
+//
+// Why a pair: a 128-row query tile with a 512-wide fp32 output fills the tensor memory of one SM, so a single
+// CTA has to recompute the scores once per output half.  With cta_group::2 and M = 128 each CTA owns 64 rows,
+// and an accumulator of N columns takes only N/2 tensor-memory columns per CTA (rows 0..63 of the CTA sit in
+// lanes 0..63 for the first N/2 columns and in lanes 64..127 for the second N/2).  O (64 x 512) then needs 256
+// columns and two score buffers 128: everything fits and every score is computed once.  The B operands are
+// split between the two CTAs' shared memories -- the 128 keys of a KV tile for S = Q K^T (64 keys each), the
+// 256 value columns of each P V instruction (128 each) -- so each K/V byte is fetched from L2 once per 128
+// query rows without any multicast copy.
+//
+// Per CTA, 7 warps:
+//   warp 0      Q and K producer (TMA), tensor-memory allocation
+//   warp 1      rank 0: the one thread that issues every MMA of the pair and the multicast commits
+//               rank 1: relay -- forwards "my Q / K / V have landed" to the leader's barriers, zero-fills the
+//               value rows of keys past the end of the sequence
+//   warps 2-5   softmax: lane l of tensor memory holds 64 score columns of row l & 63; the two threads of a row
+//               exchange their row maximum through shared memory; P goes to shared memory (K-major, 128B swizzle)
+//   warp 6      V producer (TMA) and, on rank 0, zero-fill of value rows past the end of the sequence
+// Pairs walk the work list round-robin (pair p takes items p, p + #pairs, ...), so the two CTAs of a pair agree
+// on the item sequence without exchanging anything.
+// The math per row is the paper's Eq. 1 with the causal rule, KV tile by KV tile with a running maximum.
+#pragma once
+#include "attn_mla.cuh"  // kMla* constants
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace vpp {
+
+constexpr int kMla2Threads = 224;
+constexpr int kMla2Rows = 64;                                 // query rows per CTA
+constexpr int kMla2QBytes = kMlaSlabs * kMla2Rows * 128;      // 72 KB: 9 slabs x 64 rows
+constexpr int kMla2KBytes = kMlaSlabs * 64 * 128;             // 72 KB: 9 slabs x 64 keys (this CTA's half of a tile)
+constexpr int kMla2VBytes = 2 * 2 * 2 * 64 * 128;             // 64 KB: [key half][instr][col group][64 keys][128 B]
+constexpr int kMla2PBytes = 2 * kMla2Rows * 128;              // 16 KB: 2 slabs x 64 rows
+constexpr int kMla2SmemBytes = kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes + 1024 /*align*/ + 1536;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A[smem of both] * B[smem of both]; issued by one thread of the even CTA
+__device__ __forceinline__ void mma2_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on the barrier at the same shared-memory offset in every CTA of `mask` once all MMAs issued so far are done
+__device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"(mask)
+                 : "memory");
+}
+// arrive on a barrier that lives in another CTA of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t target_rank) {
+    asm volatile(
+        "{\n\t.reg .b32 ra;\n\t"
+        "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(local_bar),
+        "r"(target_rank)
+        : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// bounded wait with cluster-scope acquire (the barrier may have been completed by the other CTA)
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    int spins = 0;
+    while (true) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((++spins & 63) == 0) {
+            if (*abort_flag != 0) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                atomicCAS(const_cast<int*>(abort_flag), 0, where);
+                return false;
+            }
+        }
+    }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMla2Threads, 1)
+attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constant__ CUtensorMap tm_k9,
+                 const __grid_constant__ CUtensorMap tm_v2, const AttnParams p) {
+    // tm_q9: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 9, 1)  -- 64 query rows, all 576 features
+    // tm_k9: (64 cols, keys, 9 slabs, head, block) box (64, 64, 9, 1, 1) -- 64 keys, all 576 features
+    // tm_v2: same tensor, box (64, 64, 2, 1, 1) -- 64 keys, two 64-column value groups
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t sQ = smem_base;
+    const uint32_t sK = sQ + kMla2QBytes;
+    const uint32_t sV = sK + kMla2KBytes;
+    const uint32_t sP = sV + kMla2VBytes;
+    const uint32_t sBar = sP + kMla2PBytes;
+    const uint32_t bar_q_full = sBar + 0, bar_q_empty = sBar + 8;
+    const uint32_t bar_k_full = sBar + 16, bar_k_empty = sBar + 24;
+    const uint32_t bar_v_full = sBar + 32, bar_v_empty = sBar + 40;
+    const uint32_t bar_s_full = sBar + 48;   // [2]
+    const uint32_t bar_p_full = sBar + 64;   // [2] (used in the leader only: 4 local + 4 remote warp arrivals)
+    const uint32_t bar_p_empty = sBar + 80;
+    const uint32_t bar_o_full = sBar + 88;
+    const uint32_t bar_vfix = sBar + 96;     // leader: V producer -> MMA thread
+    const uint32_t bar_xchg = sBar + 104;    // row statistics exchange between the two threads of a row
+    const uint32_t bar_qk_local = sBar + 112;  // rank 1: local "landed" barriers the relay waits on: q, k, v
+    uint8_t* gen_bar = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes;
+    volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 256);
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 260);
+    float* xch = reinterpret_cast<float*>(gen_bar + 512);  // [2 phases][128 lanes]
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    // rank 1 lands its copies on local barriers (bar_qk_local + 0/8/16) and its relay forwards them
+    const uint32_t my_q_full = leader ? bar_q_full : bar_qk_local;
+    const uint32_t my_k_full = leader ? bar_k_full : bar_qk_local + 8;
+    const uint32_t my_v_full = leader ? bar_v_full : bar_qk_local + 16;
+
+    if (tid == 0) {
+        mbar_init(bar_q_full, 2);   // leader: own producer + the peer's relay
+        mbar_init(bar_k_full, 2);
+        mbar_init(bar_v_full, 2);
+        mbar_init(bar_q_empty, 1);
+        mbar_init(bar_k_empty, 1);
+        mbar_init(bar_v_empty, 1);
+        mbar_init(bar_s_full, 1);
+        mbar_init(bar_s_full + 8, 1);
+        mbar_init(bar_p_full, 8);
+        mbar_init(bar_p_full + 8, 8);
+        mbar_init(bar_p_empty, 1);
+        mbar_init(bar_o_full, 1);
+        mbar_init(bar_vfix, 1);
+        mbar_init(bar_xchg, 128);
+        mbar_init(bar_qk_local, 1);
+        mbar_init(bar_qk_local + 8, 1);
+        mbar_init(bar_qk_local + 16, 1);
+        fence_mbar_init();
+        *s_abort = 0;
+        prefetch_tmap(&tm_q9);
+        prefetch_tmap(&tm_k9);
+        prefetch_tmap(&tm_v2);
+    }
+    __syncthreads();
+    cluster_sync_all();  // barrier initialisation is visible to the other CTA before anything arrives remotely
+    if (warp == 0) {
+        tmem_alloc2(smem_u32(const_cast<uint32_t*>(s_tmem)), 512);
+        tmem_relinquish2();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    const int num_units = p.header_ro->num_units;
+    const int total_items = num_units * p.num_q_heads;
+    const int num_pairs = gridDim.x >> 1;
+    const int pair = blockIdx.x >> 1;
+
+    // KV tiles (128 keys) of a unit: [kv_begin, min(kv_end, ceil((pos0 + rows) / 128)))
+    auto tile_hi = [](const WorkUnit& u) {
+        const int need = (u.pos0 + u.rows + kTileN - 1) / kTileN;
+        return u.kv_end < need ? u.kv_end : need;
+    };
+    auto get_item = [&](int item, WorkUnit& u, int& h) {
+        int ui;
+        decode_item(item, num_units, p.num_q_heads, p.num_q_heads, ui, h);
+        u = p.units[ui];
+    };
+    // page and slot of the 64-key group that starts at position pos
+    auto page_of = [&](const WorkUnit& u, int pos, int& blk, int& slot_in) {
+        if (p.block_table == nullptr) {
+            blk = u.req;
+            slot_in = pos;
+        } else if (pos < u.kv_len) {
+            blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req + (pos >> p.block_shift));
+            slot_in = pos & ((1 << p.block_shift) - 1);
+        } else {
+            blk = p.num_blocks;  // out of range: the copy engine fills zeros
+            slot_in = 0;
+        }
+    };
+
+    if (warp == 0) {
+        // ===================================== Q / K producer =====================================
+        if (lane == 0) {
+            uint32_t q_it = 0, k_it = 0;
+            for (int item = pair; item < total_items; item += num_pairs) {
+                WorkUnit u;
+                int h;
+                get_item(item, u, h);
+                if (!mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 801)) break;
+                mbar_arrive_expect_tx(my_q_full, kMla2QBytes);
+                tma_load_4d(sQ, &tm_q9, my_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, 0, h);
+                ++q_it;
+                const int t_hi = tile_hi(u);
+                bool ok = true;
+                for (int j = u.kv_begin; j < t_hi; ++j) {
+                    int blk, slot_in;
+                    page_of(u, j * kTileN + static_cast<int>(rank) * 64, blk, slot_in);
+                    ok = mbar_wait(bar_k_empty, (k_it & 1) ^ 1, s_abort, 802);
+                    if (!ok) break;
+                    mbar_arrive_expect_tx(my_k_full, kMla2KBytes);
+                    tma_load_5d(sK, &tm_k9, my_k_full, 0, slot_in, 0, 0, blk);
+                    ++k_it;
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 6) {
+        // ======================================= V producer =======================================
+        uint32_t v_it = 0;
+        bool ok = true;
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            get_item(item, u, h);
+            const int t_hi = tile_hi(u);
+            for (int j = u.kv_begin; j < t_hi && ok; ++j) {
+                const int tile0 = j * kTileN;
+                if (lane == 0) {
+                    int blk[2], slot_in[2];
+                    page_of(u, tile0, blk[0], slot_in[0]);
+                    page_of(u, tile0 + 64, blk[1], slot_in[1]);
+                    ok = mbar_wait(bar_v_empty, (v_it & 1) ^ 1, s_abort, 803);
+                    if (ok) {
+                        mbar_arrive_expect_tx(my_v_full, kMla2VBytes);
+                        // [key half][instr][2 col groups x 64 keys]; value columns of instr i for this CTA start at
+                        // slab 4 i + 2 rank
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+                                tma_load_5d(sV + (hf * 2 + i) * 16384, &tm_v2, my_v_full, 0, slot_in[hf],
+                                            4 * i + 2 * static_cast<int>(rank), 0, blk[hf]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (leader && tile0 + kTileN > u.kv_len) {
+                    // keys at or beyond kv_len do not exist: zero their value rows (0 * garbage must not reach O)
+                    if (lane == 0) ok = mbar_wait(bar_v_full, v_it & 1, s_abort, 804);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+                    for (int r = first + lane; r < kTileN; r += 32) {
+                        const int hf = r >> 6, rr = r & 63;
+#pragma unroll
+                        for (int blk4 = 0; blk4 < 4; ++blk4) {  // 2 instr x 2 col groups
+                            uint4* a = reinterpret_cast<uint4*>(gen_base + kMla2QBytes + kMla2KBytes + hf * 32768 +
+                                                                blk4 * 8192 + rr * 128);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) a[c] = z;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_vfix);
+                }
+                ++v_it;
+            }
+        }
+    } else if (warp == 1 && !leader) {
+        // ================================ relay (rank 1 only) ================================
+        uint32_t q_it = 0, kv_it = 0;
+        bool ok = true;
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            get_item(item, u, h);
+            if (lane == 0) {
+                ok = mbar_wait(bar_qk_local, q_it & 1, s_abort, 811);
+                if (ok) mbar_arrive_remote(bar_q_full, 0);
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ++q_it;
+            const int t_hi = tile_hi(u);
+            for (int j = u.kv_begin; j < t_hi && ok; ++j) {
+                const int tile0 = j * kTileN;
+                if (lane == 0) {
+                    ok = mbar_wait(bar_qk_local + 8, kv_it & 1, s_abort, 812);
+                    if (ok) mbar_arrive_remote(bar_k_full, 0);
+                    if (ok) ok = mbar_wait(bar_qk_local + 16, kv_it & 1, s_abort, 813);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (tile0 + kTileN > u.kv_len) {
+                    const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+                    for (int r = first + lane; r < kTileN; r += 32) {
+                        const int hf = r >> 6, rr = r & 63;
+#pragma unroll
+                        for (int blk4 = 0; blk4 < 4; ++blk4) {
+                            uint4* a = reinterpret_cast<uint4*>(gen_base + kMla2QBytes + kMla2KBytes + hf * 32768 +
+                                                                blk4 * 8192 + rr * 128);
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) a[c] = z;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                }
+                if (lane == 0) mbar_arrive_remote(bar_v_full, 0);
+                ++kv_it;
+            }
+        }
+    } else if (warp == 1 && leader && lane == 0) {
+        // ====================== MMA issuer: one thread for both CTAs of the pair ======================
+        constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
+        constexpr uint32_t kIdescPV = idesc_bf16(128, 256, false, true);
+        constexpr uint32_t kHi = desc_hi_sw128(1024);
+        const uint32_t q_lo = desc_lo_sw128(sQ, 16), k_lo = desc_lo_sw128(sK, 16), p_lo = desc_lo_sw128(sP, 16);
+        const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
+        const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
+        uint32_t q_it = 0, k_it = 0, v_it = 0, tc = 0, vfix_it = 0;
+        auto issue_qk = [&](uint32_t tS) {
+#pragma unroll 1
+            for (int s = 0; s < kMlaSlabs; ++s)
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma2_ss_lh(tS, q_lo + ((s * 8192 + kk * 32) >> 4), k_lo + ((s * 8192 + kk * 32) >> 4), kHi, kIdescQK,
+                               (s > 0 || kk > 0) ? 1u : 0u);
+        };
+        bool ok = true;
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            get_item(item, u, h);
+            const int n = tile_hi(u) - u.kv_begin;
+            ok = mbar_wait_cluster(bar_q_full, q_it & 1, s_abort, 821);
+            if (!ok) break;
+            ++q_it;
+            ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 822);
+            if (!ok) break;
+            ++k_it;
+            tc_fence_after();
+            issue_qk(tmem_base + (tc & 1) * 64);
+            tc_commit2(bar_k_empty, 3);
+            tc_commit2(bar_s_full + 8 * (tc & 1), 3);
+            if (n == 1) tc_commit2(bar_q_empty, 3);
+            for (int jj = 0; jj < n; ++jj) {
+                const int tile0 = (u.kv_begin + jj) * kTileN;
+                const uint32_t b = tc & 1;
+                if (jj + 1 < n) {
+                    ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 823);
+                    if (!ok) break;
+                    ++k_it;
+                    tc_fence_after();
+                    issue_qk(tmem_base + (b ^ 1) * 64);
+                    tc_commit2(bar_k_empty, 3);
+                    tc_commit2(bar_s_full + 8 * (b ^ 1), 3);
+                    if (jj + 2 == n) tc_commit2(bar_q_empty, 3);
+                }
+                ok = mbar_wait_cluster(bar_v_full, v_it & 1, s_abort, 824);
+                if (!ok) break;
+                ++v_it;
+                if (tile0 + kTileN > u.kv_len) {
+                    ok = mbar_wait(bar_vfix, vfix_it & 1, s_abort, 825);
+                    if (!ok) break;
+                    ++vfix_it;
+                }
+                ok = mbar_wait_cluster(bar_p_full + 8 * b, (tc >> 1) & 1, s_abort, 826);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        mma2_ss_lh(i == 0 ? tO0 : tO1, p_lo + (((kk >> 2) * 8192 + (kk & 3) * 32) >> 4),
+                                   v_lo + ((((kk >> 2) * 2 + i) * 16384 + (kk & 3) * 2048) >> 4), kHi, kIdescPV,
+                                   (jj > 0 || kk > 0) ? 1u : 0u);
+                tc_commit2(bar_v_empty, 3);
+                tc_commit2(bar_p_empty, 3);
+                if (jj + 1 == n) tc_commit2(bar_o_full, 3);
+                ++tc;
+            }
+        }
+    } else if (warp >= 2 && warp <= 5) {
+        // ======================================= softmax =======================================
+        const int l128 = ((warp & 3) << 5) | lane;     // TMEM lane
+        const int row = l128 & 63;                     // row of this CTA's 64
+        const int half = l128 >> 6;                    // which 64 key columns of the tile
+        const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t tO0 = tmem_base + 128 + lane_off, tO1 = tmem_base + 256 + lane_off;
+        uint8_t* p_row = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + half * 8192 + row * 128;
+        uint32_t tc = 0, o_it = 0, x_it = 0, pe_it = 0;
+        const float sc = p.scale_log2e;
+        auto exchange = [&](float mine, float& theirs) -> bool {
+            float* buf = xch + (x_it & 1) * 128;
+            buf[l128] = mine;
+            mbar_arrive(bar_xchg);
+            if (!mbar_wait(bar_xchg, x_it & 1, s_abort, 831)) return false;
+            theirs = buf[l128 ^ 64];
+            ++x_it;
+            return true;
+        };
+        bool ok = true;
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            get_item(item, u, h);
+            const int t_hi = tile_hi(u);
+            const int my_row = static_cast<int>(rank) * kMla2Rows + row;  // row of the 128-row tile
+            const int my_pos = u.pos0 + my_row;
+            float m_ref = -INFINITY, l_run = 0.f;
+            for (int j = u.kv_begin; j < t_hi; ++j) {
+                const int tile0 = j * kTileN;
+                const uint32_t b = tc & 1;
+                const uint32_t tS = tmem_base + b * 64 + lane_off;
+                ok = mbar_wait(bar_s_full + 8 * b, (tc >> 1) & 1, s_abort, 832);
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t s[64];
+                tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
+                tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
+                tc_wait_ld();
+                if (tile0 + kTileN - 1 > u.pos0) {  // diagonal tile
+                    const int lim = my_pos - tile0 - half * 64;
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        if (i > lim) s[i] = 0xff800000u;  // -inf
+                }
+                float mx[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) mx[k] = __uint_as_float(s[k]);
+#pragma unroll
+                for (int i = 8; i < 64; i += 8)
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) mx[k] = fmaxf(mx[k], __uint_as_float(s[i + k]));
+                const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                        fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                float mxb;
+                ok = exchange(mxa, mxb);
+                if (!ok) break;
+                const float m_new = fmaxf(fmaxf(mxa, mxb) * sc, m_ref);
+                const bool grow = (m_new - m_ref > 8.f) || (m_ref == -INFINITY && m_new != -INFINITY);
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float alpha = grow ? ex2(m_ref - m_new) : 1.f;
+                    if (grow) m_ref = m_new;
+                    l_run *= alpha;
+                    if (j > u.kv_begin) {
+                        uint32_t o[32];
+#pragma unroll 1
+                        for (int c = 0; c < 8; ++c) {
+                            const uint32_t addr = (c < 4 ? tO0 : tO1) + (c & 3) * 32;
+                            tmem_ld32(addr, o);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(addr, o);
+                        }
+                        tc_wait_st();
+                    }
+                }
+                const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+                uint32_t pk[32];
+                float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 64; i += 2) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s[i]), sc, -m_use));
+                    const float p1 = ex2(fmaf(__uint_as_float(s[i + 1]), sc, -m_use));
+                    sum0 += p0;
+                    sum1 += p1;
+                    pk[i >> 1] = pack_bf16x2(p0, p1);
+                }
+                l_run += sum0 + sum1;
+                // P of the previous tile must have been consumed before its shared-memory rows are overwritten
+                if (tc > 0) {
+                    ok = mbar_wait(bar_p_empty, pe_it & 1, s_abort, 833);
+                    if (!ok) break;
+                    ++pe_it;
+                }
+#pragma unroll
+                for (int c = 0; c < 8; ++c)  // K-major 128B-swizzled row: 16-byte chunk index XOR (row & 7)
+                    *reinterpret_cast<uint4*>(p_row + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                fence_proxy_async_smem();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (leader) mbar_arrive(bar_p_full + 8 * b);
+                    else mbar_arrive_remote(bar_p_full + 8 * b, 0);
+                }
+                ++tc;
+            }
+            if (!ok) break;
+            // ---- epilogue ----
+            float l_other;
+            ok = exchange(l_run, l_other);
+            if (!ok) break;
+            const float l_tot = l_run + l_other;
+            ok = mbar_wait(bar_o_full, o_it & 1, s_abort, 834);
+            if (!ok) break;
+            ++o_it;
+            tc_fence_after();
+            const float inv_l = 1.f / l_tot;
+            const bool live = my_row < u.rows;
+            const long long grow_idx = static_cast<long long>(u.q_row0) + my_row;
+            uint32_t r[32];
+#pragma unroll 1
+            for (int c = 0; c < 8; ++c) {
+                tmem_ld32((c < 4 ? tO0 : tO1) + (c & 3) * 32, r);
+                tc_wait_ld();
+                if (!live) continue;
+                const int col0 = (c >> 2) * 256 + half * 128 + (c & 3) * 32;
+                if (u.split < 0) {
+                    uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                          ((grow_idx * p.num_q_heads + h) * kMlaDv + col0) * 2);
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            w[e] = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2 * e]) * inv_l,
+                                               __uint_as_float(r[q4 * 8 + 2 * e + 1]) * inv_l);
+                        dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                } else {
+                    float4* dst = reinterpret_cast<float4*>(
+                        p.o_parts + ((static_cast<long long>(u.split) * p.total_q + grow_idx) * p.num_q_heads + h) * kMlaDv +
+                        col0);
+#pragma unroll
+                    for (int q4 = 0; q4 < 8; ++q4)
+                        dst[q4] = make_float4(__uint_as_float(r[q4 * 4]) * inv_l, __uint_as_float(r[q4 * 4 + 1]) * inv_l,
+                                              __uint_as_float(r[q4 * 4 + 2]) * inv_l, __uint_as_float(r[q4 * 4 + 3]) * inv_l);
+                }
+            }
+            if (live && half == 0) {
+                const float lse = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+                if (u.split < 0) {
+                    if (p.lse) p.lse[grow_idx * p.num_q_heads + h] = lse;
+                } else {
+                    p.lse_parts[(static_cast<long long>(u.split) * p.total_q + grow_idx) * p.num_q_heads + h] = lse;
+                }
+            }
+            tc_fence_before();
+        }
+    }
+
+    // ---- teardown ----
+    __syncthreads();
+    if (*s_abort != 0) {
+        if (tid == 0 && p.status) atomicCAS(p.status, 0, 3 /* VPP_DEV_TIMEOUT */);
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // neither CTA frees tensor memory or exits while the other may still signal it
+    if (warp == 0) tmem_dealloc2(tmem_base, 512);
+}
+
+}  // namespace vpp
