@@ -322,22 +322,20 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_k2, a->k_cache, 5, d, sk, b5) || !make_tmap(&tm_v2, a->v_cache, 5, d, sv, b5))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
     }
-    CUtensorMap tm_q9, tm_k9, tm_v2m;
+    CUtensorMap tm_q9, tm_k9;  // one 64-column slab of 64 rows per box
     const bool mla_pair = fam == Family::kMla576 && use_mla_pair_kernel(a);
     if (mla_pair) {
         const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), static_cast<uint64_t>(vpp::kMlaSlabs),
                                 static_cast<uint64_t>(a->num_q_heads)};
         const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
                                 static_cast<uint64_t>(a->head_dim_qk) * 2};
-        const uint32_t bq[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};
+        const uint32_t bq[4] = {64, 64, 1, 1};
         const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
                                static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
         const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
                                 static_cast<uint64_t>(a->k_block_stride) * 2};
-        const uint32_t b9[5] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1, 1};
-        const uint32_t b2[5] = {64, 64, 2, 1, 1};
-        if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) || !make_tmap(&tm_k9, a->k_cache, 5, d, sk, b9) ||
-            !make_tmap(&tm_v2m, a->k_cache, 5, d, sk, b2))
+        const uint32_t b1[5] = {64, 64, 1, 1, 1};
+        if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) || !make_tmap(&tm_k9, a->k_cache, 5, d, sk, b1))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");
     }
     CUtensorMap tm_k4, tm_k5;
@@ -403,7 +401,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     if (mla_pair) {
         auto kern = vpp::attn_mla2_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
-        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, tm_v2m, ap);
+        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, ap);
     } else if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);

@@ -67,6 +67,9 @@ __device__ __forceinline__ void mma2_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint3
         "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+#ifdef VPP_T_NO_MMA   // timing experiment only: results are wrong
+#define mma2_ss_lh(...) do {} while (0)
+#endif
 // arrive on the barrier at the same shared-memory offset in every CTA of `mask` once all MMAs issued so far are done
 __device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t mask) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
@@ -100,6 +103,9 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
     int spins = 0;
     while (true) {
         if (mbar_try_wait_cluster(bar, parity)) return true;
+#ifdef VPP_WAIT_SLEEP
+        __nanosleep(VPP_WAIT_SLEEP);
+#endif
         if ((++spins & 63) == 0) {
             if (*abort_flag != 0) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
@@ -111,11 +117,12 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMla2Threads, 1)
-attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constant__ CUtensorMap tm_k9,
-                 const __grid_constant__ CUtensorMap tm_v2, const AttnParams p) {
-    // tm_q9: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 9, 1)  -- 64 query rows, all 576 features
-    // tm_k9: (64 cols, keys, 9 slabs, head, block) box (64, 64, 9, 1, 1) -- 64 keys, all 576 features
-    // tm_v2: same tensor, box (64, 64, 2, 1, 1) -- 64 keys, two 64-column value groups
+attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_k1,
+                 const AttnParams p) {
+    // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 1, 1)         -- 64 query rows of one 64-column slab
+    // tm_k1: (64 cols, keys, 9 slabs, head, block) box (64, 64, 1, 1, 1) -- 64 keys of one 64-column slab
+    // One copy instruction moves data at only ~15 B/clk; bandwidth comes from many copies in flight, so every
+    // tile is fetched slab by slab with one copy per lane of the producer warp.
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -169,9 +176,8 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
         mbar_init(bar_qk_local + 16, 1);
         fence_mbar_init();
         *s_abort = 0;
-        prefetch_tmap(&tm_q9);
-        prefetch_tmap(&tm_k9);
-        prefetch_tmap(&tm_v2);
+        prefetch_tmap(&tm_q1);
+        prefetch_tmap(&tm_k1);
     }
     __syncthreads();
     cluster_sync_all();  // barrier initialisation is visible to the other CTA before anything arrives remotely
@@ -215,57 +221,73 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
 
     if (warp == 0) {
         // ===================================== Q / K producer =====================================
-        if (lane == 0) {
-            uint32_t q_it = 0, k_it = 0;
-            for (int item = pair; item < total_items; item += num_pairs) {
-                WorkUnit u;
-                int h;
-                get_item(item, u, h);
-                if (!mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 801)) break;
-                mbar_arrive_expect_tx(my_q_full, kMla2QBytes);
-                tma_load_4d(sQ, &tm_q9, my_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, 0, h);
-                ++q_it;
-                const int t_hi = tile_hi(u);
-                bool ok = true;
-                for (int j = u.kv_begin; j < t_hi; ++j) {
-                    int blk, slot_in;
-                    page_of(u, j * kTileN + static_cast<int>(rank) * 64, blk, slot_in);
-                    ok = mbar_wait(bar_k_empty, (k_it & 1) ^ 1, s_abort, 802);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(my_k_full, kMla2KBytes);
-                    tma_load_5d(sK, &tm_k9, my_k_full, 0, slot_in, 0, 0, blk);
-                    ++k_it;
-                }
-                if (!ok) break;
-            }
-        }
-    } else if (warp == 6) {
-        // ======================================= V producer =======================================
-        uint32_t v_it = 0;
+        // lane s < 9 copies slab s; lane 0 also posts the expected byte count and does the page lookup
+        uint32_t q_it = 0, k_it = 0, item_it = 0;
         bool ok = true;
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
             get_item(item, u, h);
+            ++item_it;
+            if (lane == 0) {
+                ok = mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 801);
+                if (ok) mbar_arrive_expect_tx(my_q_full, kMla2QBytes);
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            if (lane < kMlaSlabs)
+                tma_load_4d(sQ + lane * 8192, &tm_q1, my_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, lane, h);
+            ++q_it;
+            const int t_hi = tile_hi(u);
+            for (int j = u.kv_begin; j < t_hi; ++j) {
+                int blk = 0, slot_in = 0;
+                if (lane == 0) {
+                    page_of(u, j * kTileN + static_cast<int>(rank) * 64, blk, slot_in);
+                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 0);
+                    ok = mbar_wait(bar_k_empty, (k_it & 1) ^ 1, s_abort, 802);
+                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 1);
+                    if (ok) mbar_arrive_expect_tx(my_k_full, kMla2KBytes);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                blk = __shfl_sync(0xffffffffu, blk, 0);
+                slot_in = __shfl_sync(0xffffffffu, slot_in, 0);
+                if (lane < kMlaSlabs) tma_load_5d(sK + lane * 8192, &tm_k1, my_k_full, 0, slot_in, lane, 0, blk);
+                if (lane == 0) VPP_TR(3, j - u.kv_begin, 2);
+                if (lane == 0) VPP_TR1(2, j - u.kv_begin, 2);
+                ++k_it;
+            }
+        }
+    } else if (warp == 6) {
+        // ======================================= V producer =======================================
+        uint32_t v_it = 0, item_it = 0;
+        bool ok = true;
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            get_item(item, u, h);
+            ++item_it;
             const int t_hi = tile_hi(u);
             for (int j = u.kv_begin; j < t_hi && ok; ++j) {
                 const int tile0 = j * kTileN;
+                int blk = 0, slot_in = 0;
+                if (lane < 2) page_of(u, tile0 + 64 * lane, blk, slot_in);   // lane hf looks up key half hf
                 if (lane == 0) {
-                    int blk[2], slot_in[2];
-                    page_of(u, tile0, blk[0], slot_in[0]);
-                    page_of(u, tile0 + 64, blk[1], slot_in[1]);
+                    VPP_TR(3, j - u.kv_begin, 3);
                     ok = mbar_wait(bar_v_empty, (v_it & 1) ^ 1, s_abort, 803);
-                    if (ok) {
-                        mbar_arrive_expect_tx(my_v_full, kMla2VBytes);
-                        // [key half][instr][2 col groups x 64 keys]; value columns of instr i for this CTA start at
-                        // slab 4 i + 2 rank
-#pragma unroll
-                        for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                            for (int i = 0; i < 2; ++i)
-                                tma_load_5d(sV + (hf * 2 + i) * 16384, &tm_v2, my_v_full, 0, slot_in[hf],
-                                            4 * i + 2 * static_cast<int>(rank), 0, blk[hf]);
-                    }
+                    VPP_TR(3, j - u.kv_begin, 4);
+                    if (ok) mbar_arrive_expect_tx(my_v_full, kMla2VBytes);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (ok) {
+                    // lane = hf*4 + i*2 + g copies value group g of instr i for key half hf: slab 4 i + 2 rank + g,
+                    // to [key half][instr][col group][64 keys][128 B]
+                    const int hf = (lane >> 2) & 1, ig = lane & 3;
+                    const int b2 = __shfl_sync(0xffffffffu, blk, hf), s2 = __shfl_sync(0xffffffffu, slot_in, hf);
+                    if (lane < 8)
+                        tma_load_5d(sV + lane * 8192, &tm_k1, my_v_full, 0, s2, 4 * (ig >> 1) + 2 * static_cast<int>(rank) + (ig & 1),
+                                    0, b2);
+                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 5);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
@@ -295,12 +317,13 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
         }
     } else if (warp == 1 && !leader) {
         // ================================ relay (rank 1 only) ================================
-        uint32_t q_it = 0, kv_it = 0;
+        uint32_t q_it = 0, kv_it = 0, item_it = 0;
         bool ok = true;
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
             get_item(item, u, h);
+            ++item_it;
             if (lane == 0) {
                 ok = mbar_wait(bar_qk_local, q_it & 1, s_abort, 811);
                 if (ok) mbar_arrive_remote(bar_q_full, 0);
@@ -312,8 +335,10 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                 const int tile0 = j * kTileN;
                 if (lane == 0) {
                     ok = mbar_wait(bar_qk_local + 8, kv_it & 1, s_abort, 812);
+                    VPP_TR1(2, j - u.kv_begin, 0);
                     if (ok) mbar_arrive_remote(bar_k_full, 0);
                     if (ok) ok = mbar_wait(bar_qk_local + 16, kv_it & 1, s_abort, 813);
+                    VPP_TR1(2, j - u.kv_begin, 1);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
@@ -345,7 +370,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
         const uint32_t q_lo = desc_lo_sw128(sQ, 16), k_lo = desc_lo_sw128(sK, 16), p_lo = desc_lo_sw128(sP, 16);
         const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
         const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
-        uint32_t q_it = 0, k_it = 0, v_it = 0, tc = 0, vfix_it = 0;
+        uint32_t q_it = 0, k_it = 0, v_it = 0, tc = 0, vfix_it = 0, item_it = 0;
         auto issue_qk = [&](uint32_t tS) {
 #pragma unroll 1
             for (int s = 0; s < kMlaSlabs; ++s)
@@ -360,6 +385,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
             int h;
             get_item(item, u, h);
             const int n = tile_hi(u) - u.kv_begin;
+            ++item_it;
             ok = mbar_wait_cluster(bar_q_full, q_it & 1, s_abort, 821);
             if (!ok) break;
             ++q_it;
@@ -374,19 +400,28 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
             for (int jj = 0; jj < n; ++jj) {
                 const int tile0 = (u.kv_begin + jj) * kTileN;
                 const uint32_t b = tc & 1;
-                if (jj + 1 < n) {
-                    ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 823);
-                    if (!ok) break;
+                VPP_TR(0, jj, 0);
+                // Scores of the next tile first if its keys are already here (they overlap this tile's softmax);
+                // otherwise P V of this tile goes first so that the tensor core is not idle while the keys arrive.
+                auto next_scores = [&]() {
                     ++k_it;
                     tc_fence_after();
+                    VPP_TR(0, jj, 1);
                     issue_qk(tmem_base + (b ^ 1) * 64);
+                    VPP_TR(0, jj, 2);
                     tc_commit2(bar_k_empty, 3);
                     tc_commit2(bar_s_full + 8 * (b ^ 1), 3);
                     if (jj + 2 == n) tc_commit2(bar_q_empty, 3);
+                };
+                bool scores_done = jj + 1 >= n;
+                if (!scores_done && mbar_try_wait_cluster(bar_k_full, k_it & 1)) {
+                    next_scores();
+                    scores_done = true;
                 }
                 ok = mbar_wait_cluster(bar_v_full, v_it & 1, s_abort, 824);
                 if (!ok) break;
                 ++v_it;
+                VPP_TR(0, jj, 3);
                 if (tile0 + kTileN > u.kv_len) {
                     ok = mbar_wait(bar_vfix, vfix_it & 1, s_abort, 825);
                     if (!ok) break;
@@ -395,6 +430,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                 ok = mbar_wait_cluster(bar_p_full + 8 * b, (tc >> 1) & 1, s_abort, 826);
                 if (!ok) break;
                 tc_fence_after();
+                VPP_TR(0, jj, 4);
 #pragma unroll
                 for (int i = 0; i < 2; ++i)
 #pragma unroll
@@ -404,7 +440,13 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                                    (jj > 0 || kk > 0) ? 1u : 0u);
                 tc_commit2(bar_v_empty, 3);
                 tc_commit2(bar_p_empty, 3);
+                VPP_TR(0, jj, 5);
                 if (jj + 1 == n) tc_commit2(bar_o_full, 3);
+                if (!scores_done) {
+                    ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 823);
+                    if (!ok) break;
+                    next_scores();
+                }
                 ++tc;
             }
         }
@@ -416,7 +458,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tO0 = tmem_base + 128 + lane_off, tO1 = tmem_base + 256 + lane_off;
         uint8_t* p_row = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + half * 8192 + row * 128;
-        uint32_t tc = 0, o_it = 0, x_it = 0, pe_it = 0;
+        uint32_t tc = 0, o_it = 0, x_it = 0, pe_it = 0, item_it = 0;
         const float sc = p.scale_log2e;
         auto exchange = [&](float mine, float& theirs) -> bool {
             float* buf = xch + (x_it & 1) * 128;
@@ -433,6 +475,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
             int h;
             get_item(item, u, h);
             const int t_hi = tile_hi(u);
+            ++item_it;
             const int my_row = static_cast<int>(rank) * kMla2Rows + row;  // row of the 128-row tile
             const int my_pos = u.pos0 + my_row;
             float m_ref = -INFINITY, l_run = 0.f;
@@ -443,6 +486,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                 ok = mbar_wait(bar_s_full + 8 * b, (tc >> 1) & 1, s_abort, 832);
                 if (!ok) break;
                 tc_fence_after();
+                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 0);
                 uint32_t s[64];
                 tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                 tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
@@ -463,8 +507,10 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                 const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 float mxb;
+                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 1);
                 ok = exchange(mxa, mxb);
                 if (!ok) break;
+                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 2);
                 const float m_new = fmaxf(fmaxf(mxa, mxb) * sc, m_ref);
                 const bool grow = (m_new - m_ref > 8.f) || (m_ref == -INFINITY && m_new != -INFINITY);
                 if (__any_sync(0xffffffffu, grow)) {
@@ -497,6 +543,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                     pk[i >> 1] = pack_bf16x2(p0, p1);
                 }
                 l_run += sum0 + sum1;
+                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 3);
                 // P of the previous tile must have been consumed before its shared-memory rows are overwritten
                 if (tc > 0) {
                     ok = mbar_wait(bar_p_empty, pe_it & 1, s_abort, 833);
@@ -510,6 +557,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q9, const __grid_constan
                 fence_proxy_async_smem();
                 tc_fence_before();
                 __syncwarp();
+                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 4);
                 if (lane == 0) {
                     if (leader) mbar_arrive(bar_p_full + 8 * b);
                     else mbar_arrive_remote(bar_p_full + 8 * b, 0);

@@ -66,8 +66,13 @@ __device__ long long g_trace[64 * 32];
     do {                                                                                        \
         if (blockIdx.x == 0 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
     } while (0)
+#define VPP_TR1(role, jj, k)                                                                    \
+    do {                                                                                        \
+        if (blockIdx.x == 1 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
+    } while (0)
 #else
 #define VPP_TR(role, jj, k) do {} while (0)
+#define VPP_TR1(role, jj, k) do {} while (0)
 #endif
 
 }  // namespace vpp

@@ -59,6 +59,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     int spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
+#ifdef VPP_WAIT_SLEEP
+        __nanosleep(VPP_WAIT_SLEEP);
+#endif
         if ((++spins & 63) == 0) {
             if (*abort_flag != 0) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
@@ -103,6 +106,14 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* m, 
         "[%2];" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
+}
+
+// L2 prefetch of a rank-5 box (no shared-memory destination, no barrier)
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* m, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global [%0, {%1, %2, %3, %4, %5}];" ::"l"(
+                     reinterpret_cast<uint64_t>(m)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+                 : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
