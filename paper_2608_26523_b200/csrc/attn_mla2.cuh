@@ -67,9 +67,6 @@ __device__ __forceinline__ void mma2_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint3
         "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-#ifdef VPP_T_NO_MMA   // timing experiment only: results are wrong
-#define mma2_ss_lh(...) do {} while (0)
-#endif
 // arrive on the barrier at the same shared-memory offset in every CTA of `mask` once all MMAs issued so far are done
 __device__ __forceinline__ void tc_commit2(uint32_t bar, uint16_t mask) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
