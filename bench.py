@@ -142,6 +142,8 @@ def main():
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--max-prefix", type=int, default=0,
+                    help="size the KV cache (and its page pool) for this prefix even if the run uses shorter ones")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -210,7 +212,7 @@ def main():
         D.init("nccl", dev)
     api.load_library()
 
-    max_prefix = max(prefixes)
+    max_prefix = max(max(prefixes), args.max_prefix)
     stream = torch.cuda.Stream(device=dev)
     runners = []
     if args.workload == "cfg5":

@@ -32,6 +32,12 @@ constexpr int kWsStages = VPP_WS_STAGES;      // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 1024 /*barriers, ring*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
+#ifndef VPP_SPLIT_CHUNKS
+#define VPP_SPLIT_CHUNKS 1
+#endif
+// 0: P is handed to the MMA thread whole; c in 1..3: the first 32*c key columns are handed over early so that
+// O += P V can start on them while the rest of the exponentials are computed
+constexpr int kSplitChunks = VPP_SPLIT_CHUNKS;
 #ifndef VPP_EMU_EVERY
 #define VPP_EMU_EVERY 0
 #endif
@@ -69,6 +75,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_p_full = sBar + 64;       // [2]
     const uint32_t bar_o_full = sBar + 80;       // [2]
     const uint32_t bar_vfix = sBar + 96;
+    const uint32_t bar_p_part = sBar + 104;      // [2] first kSplitCols key columns of P are in place (optional early hand-off)
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
     const uint32_t bar_kv_empty = sBar + 128 + 8 * kWsStages;
     uint8_t* gen_bar = gen_base + (2 + kWsStages) * kTileBytes;
@@ -86,6 +93,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(bar_item_empty + 8 * i, 9);
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_p_full + 8 * i, 4);   // one arrival per softmax warp
+            mbar_init(bar_p_part + 8 * i, 4);
             mbar_init(bar_o_full + 8 * i, 1);
         }
         mbar_init(bar_q_full, 1);
@@ -325,11 +333,24 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const bool has_next = jj + 1 < n;
                     stK = kv_it % kWsStages;
                     // ---- tile 0 ----
-                    ok = wait1(bar_p_full, p_it & 1, 306);
-                    if (!ok) break;
-                    tc_fence_after();
+                    if (kSplitChunks == 0) {
+                        ok = wait1(bar_p_full, p_it & 1, 306);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
                     if (lane == 0) VPP_TR(0, jj, 1);
-                    issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
+                    if (kSplitChunks > 0) {
+                        ok = wait1(bar_p_part, p_it & 1, 311);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 2 * kSplitChunks);
+                        ok = wait1(bar_p_full, p_it & 1, 306);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 2 * kSplitChunks, 8);
+                    } else {
+                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
+                    }
                     if (lane == 0) VPP_TR(0, jj, 2);
                     if (has_next) {
 #ifdef VPP_TRACE
@@ -354,12 +375,18 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         tc_commit(bar_o_full);
                     }
                     // ---- tile 1 ----
+                    if (kSplitChunks > 0) {
+                        ok = wait1(bar_p_part + 8, p_it & 1, 312);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 2 * kSplitChunks);
+                    }
                     ok = wait1(bar_p_full + 8, p_it & 1, 308);
                     if (!ok) break;
                     tc_fence_after();
                     if (lane == 0) VPP_TR(0, jj, 5);
                     if (lane == 0) {
-                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 8);
+                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, kSplitChunks > 0 ? 2 * kSplitChunks : 0, 8);
                         tc_commit(bar_kv_empty + 8 * stV);
                         if (has_next) {
                             issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
@@ -490,6 +517,12 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         pk[i >> 1] = pack_bf16x2(p0, p1);
                     }
                     tmem_st16(tS + c * 16, pk);
+                    if (kSplitChunks > 0 && c == kSplitChunks - 1) {
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_p_part + 8 * t);
+                    }
                 }
                 l_run += sum0 + sum1;
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 3);
