@@ -11,13 +11,19 @@
 // query rows without any multicast copy.
 //
 // Per CTA, 7 warps:
-//   warp 0      Q and K producer (TMA), tensor-memory allocation
-//   warp 1      rank 0: the one thread that issues every MMA of the pair and the multicast commits
-//               rank 1: relay -- forwards "my Q / K / V have landed" to the leader's barriers, zero-fills the
-//               value rows of keys past the end of the sequence
+//   warp 0      one thread: Q and K producer (TMA); the warp also allocates tensor memory
+//   warp 1      rank 0: the one thread that issues every MMA of the pair and the multicast commits; rank 1: idle
 //   warps 2-5   softmax: lane l of tensor memory holds 64 score columns of row l & 63; the two threads of a row
 //               exchange their row maximum through shared memory; P goes to shared memory (K-major, 128B swizzle)
-//   warp 6      V producer (TMA) and, on rank 0, zero-fill of value rows past the end of the sequence
+//   warp 6      V producer (TMA) and zero-fill of value rows past the end of the sequence
+// Copies issued by either CTA post their bytes on the leader's barriers (cp.async.bulk.tensor with cta_group::2,
+// no multicast), so the MMA thread waits on local barriers only.
+//
+// What bounds the loop is the single issuing thread and the tensor pipe's fixed costs, measured on a B200:
+// a tcgen05.mma of this shape occupies the pipe for at least ~48 clk (N = 128) or ~67 clk (N = 256), and every
+// tcgen05.commit adds a bubble of ~90 clk.  Hence few commits (five per KV tile), each doubling as several
+// signals, and K / V handed back to the producers in groups (3 x 3 slabs, 2 x 32 KB) so that the copy of the
+// next tile overlaps the MMAs of this one although shared memory holds only one K and one V tile.
 // Pairs walk the work list round-robin (pair p takes items p, p + #pairs, ...), so the two CTAs of a pair agree
 // on the item sequence without exchanging anything.
 // The math per row is the paper's Eq. 1 with the causal rule, KV tile by KV tile with a running maximum.
@@ -34,6 +40,11 @@ constexpr int kMla2QBytes = kMlaSlabs * kMla2Rows * 128;      // 72 KB: 9 slabs 
 constexpr int kMla2KBytes = kMlaSlabs * 64 * 128;             // 72 KB: 9 slabs x 64 keys (this CTA's half of a tile)
 constexpr int kMla2VBytes = 2 * 2 * 2 * 64 * 128;             // 64 KB: [key half][instr][col group][64 keys][128 B]
 constexpr int kMla2PBytes = 2 * kMla2Rows * 128;              // 16 KB: 2 slabs x 64 rows
+constexpr int kMla2VChunks = 4;                               // V is refilled in 16 KB chunks: (key half, instr)
+constexpr int kMla2VChunk = kMla2VBytes / kMla2VChunks;
+constexpr int kKG = 3;  // K slabs per hand-back group (3 groups per tile)
+constexpr int kVG = 2;  // V chunks per hand-back group (2 groups per tile: key half 0, key half 1)
+constexpr int kKGroups = kMlaSlabs / kKG, kVGroups = kMla2VChunks / kVG;
 constexpr int kMla2SmemBytes = kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes + 1024 /*align*/ + 1536;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -78,8 +89,37 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t local_bar, uint32_t 
     asm volatile(
         "{\n\t.reg .b32 ra;\n\t"
         "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
-        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(local_bar),
+        #ifdef VPP_T2_ARRIVE_CLUSTER
+        "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}"
+#else
+        "mbarrier.arrive.shared::cluster.b64 _, [ra];\n\t}"
+#endif
+ ::"r"(local_bar),
         "r"(target_rank)
+        : "memory");
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Tiled copies of a CTA pair: the data lands in the executing CTA's shared memory, the byte count is posted on a
+// barrier that may live in the other CTA of the pair (bar_cluster is a shared::cluster address).  No multicast.
+__device__ __forceinline__ void tma2_load_4d(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1,
+                                             int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, "
+        "%6}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma2_load_5d(uint32_t dst, const CUtensorMap* m, uint32_t bar_cluster, int c0, int c1,
+                                             int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, "
+        "%6, %7}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(m)), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
@@ -118,8 +158,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                  const AttnParams p) {
     // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 1, 1)         -- 64 query rows of one 64-column slab
     // tm_k1: (64 cols, keys, 9 slabs, head, block) box (64, 64, 1, 1, 1) -- 64 keys of one 64-column slab
-    // One copy instruction moves data at only ~15 B/clk; bandwidth comes from many copies in flight, so every
-    // tile is fetched slab by slab with one copy per lane of the producer warp.
+    // Every tile is fetched slab by slab (8 KB copies).
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -128,19 +167,25 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
     const uint32_t sV = sK + kMla2KBytes;
     const uint32_t sP = sV + kMla2VBytes;
     const uint32_t sBar = sP + kMla2PBytes;
-    const uint32_t bar_q_full = sBar + 0, bar_q_empty = sBar + 8;
-    const uint32_t bar_k_full = sBar + 16, bar_k_empty = sBar + 24;
-    const uint32_t bar_v_full = sBar + 32, bar_v_empty = sBar + 40;
-    const uint32_t bar_s_full = sBar + 48;   // [2]
-    const uint32_t bar_p_full = sBar + 64;   // [2] (used in the leader only: 4 local + 4 remote warp arrivals)
-    const uint32_t bar_p_empty = sBar + 80;
-    const uint32_t bar_o_full = sBar + 88;
-    const uint32_t bar_vfix = sBar + 96;     // leader: V producer -> MMA thread
-    const uint32_t bar_xchg = sBar + 104;    // row statistics exchange between the two threads of a row
-    const uint32_t bar_qk_local = sBar + 112;  // rank 1: local "landed" barriers the relay waits on: q, k, v
+    // A tcgen05.commit costs the tensor pipe about as much as two small MMAs, so there are as few as possible: one
+    // per K group, the last of which doubles as "scores ready", and one per V group, the last of which doubles as
+    // "P consumed" and "O complete".  A barrier may have any number of waiters.
+    const uint32_t bar_q_full = sBar + 0;
+    const uint32_t bar_pv_done = sBar + 8;   // all P V MMAs of a tile done: last V group free, P free, O quiescent
+    const uint32_t bar_s_full = sBar + 24;   // [2] scores of a tile done: also "last K group free" (and Q free after an item)
+    const uint32_t bar_p_full = sBar + 40;   // [2] (used in the leader only: 4 local + 4 remote warp arrivals)
+    const uint32_t bar_vfix = sBar + 72;     // leader: both V producers -> MMA thread (tiles past the end of a sequence)
+    const uint32_t bar_xchg = sBar + 80;     // row statistics exchange between the two threads of a row
+    // K and V are refilled piecewise: the copy of the next tile's group starts as soon as the MMAs that read this
+    // tile's group have finished
+    const uint32_t bar_k_full = sBar + 96;    // [kKGroups] leader: bytes of both CTAs
+    const uint32_t bar_k_empty = sBar + 168;  // [kKGroups - 1]
+    const uint32_t bar_v_full = sBar + 312;   // [kVGroups]
+    const uint32_t bar_v_empty = sBar + 344;  // [kVGroups - 1]
+    const uint32_t bar_v_local = sBar + 376;  // [kVGroups] rank 1: tiles past the end of the sequence land here
     uint8_t* gen_bar = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes;
-    volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 256);
-    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 260);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 416);
+    volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 420);
     float* xch = reinterpret_cast<float*>(gen_bar + 512);  // [2 phases][128 lanes]
 
     const int tid = threadIdx.x;
@@ -148,29 +193,24 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
     const int lane = tid & 31;
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
-    // rank 1 lands its copies on local barriers (bar_qk_local + 0/8/16) and its relay forwards them
-    const uint32_t my_q_full = leader ? bar_q_full : bar_qk_local;
-    const uint32_t my_k_full = leader ? bar_k_full : bar_qk_local + 8;
-    const uint32_t my_v_full = leader ? bar_v_full : bar_qk_local + 16;
-
     if (tid == 0) {
-        mbar_init(bar_q_full, 2);   // leader: own producer + the peer's relay
-        mbar_init(bar_k_full, 2);
-        mbar_init(bar_v_full, 2);
-        mbar_init(bar_q_empty, 1);
-        mbar_init(bar_k_empty, 1);
-        mbar_init(bar_v_empty, 1);
+        mbar_init(bar_q_full, 1);
+        mbar_init(bar_pv_done, 1);
         mbar_init(bar_s_full, 1);
         mbar_init(bar_s_full + 8, 1);
         mbar_init(bar_p_full, 8);
         mbar_init(bar_p_full + 8, 8);
-        mbar_init(bar_p_empty, 1);
-        mbar_init(bar_o_full, 1);
-        mbar_init(bar_vfix, 1);
+        mbar_init(bar_vfix, 2);     // one arrival per CTA
         mbar_init(bar_xchg, 128);
-        mbar_init(bar_qk_local, 1);
-        mbar_init(bar_qk_local + 8, 1);
-        mbar_init(bar_qk_local + 16, 1);
+        for (int i = 0; i < kKGroups; ++i) {
+            mbar_init(bar_k_full + 8 * i, 1);
+            mbar_init(bar_k_empty + 8 * i, 1);
+        }
+        for (int i = 0; i < kVGroups; ++i) {
+            mbar_init(bar_v_full + 8 * i, 1);
+            mbar_init(bar_v_empty + 8 * i, 1);
+            mbar_init(bar_v_local + 8 * i, 1);
+        }
         fence_mbar_init();
         *s_abort = 0;
         prefetch_tmap(&tm_q1);
@@ -216,147 +256,139 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         }
     };
 
+    // zero the value rows of keys at or beyond `first` (position within the tile) in V chunk c = (key half, instr)
+    auto zero_v_rows = [&](int c, int first) {
+        const int r0 = first - (c >> 1) * 64;
+        const uint4 z = make_uint4(0, 0, 0, 0);
+        for (int rr = (r0 > 0 ? r0 : 0) + lane; rr < 64; rr += 32) {
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                uint4* a = reinterpret_cast<uint4*>(gen_base + kMla2QBytes + kMla2KBytes + c * kMla2VChunk + g * 8192 +
+                                                    rr * 128);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) a[q] = z;
+            }
+        }
+    };
+
+    // Copies of both CTAs post their bytes on the leader's "full" barriers (the MMA thread lives there); the leader's
+    // producer announces the byte count of the pair.  Each CTA waits on its own "empty" barriers (multicast commits).
+    const uint32_t pair_q_full = mapa_u32(bar_q_full, 0), pair_k_full = mapa_u32(bar_k_full, 0),
+                   pair_v_full = mapa_u32(bar_v_full, 0);
+
     if (warp == 0) {
         // ===================================== Q / K producer =====================================
-        // lane s < 9 copies slab s; lane 0 also posts the expected byte count and does the page lookup
-        uint32_t q_it = 0, k_it = 0, item_it = 0;
-        bool ok = true;
-        for (int item = pair; item < total_items && ok; item += num_pairs) {
-            WorkUnit u;
-            int h;
-            get_item(item, u, h);
-            ++item_it;
-            if (lane == 0) {
-                ok = mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 801);
-                if (ok) mbar_arrive_expect_tx(my_q_full, kMla2QBytes);
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            if (!ok) break;
-            if (lane < kMlaSlabs)
-                tma_load_4d(sQ + lane * 8192, &tm_q1, my_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, lane, h);
-            ++q_it;
-            const int t_hi = tile_hi(u);
-            for (int j = u.kv_begin; j < t_hi; ++j) {
-                int blk = 0, slot_in = 0;
-                if (lane == 0) {
-                    page_of(u, j * kTileN + static_cast<int>(rank) * 64, blk, slot_in);
-                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 0);
-                    ok = mbar_wait(bar_k_empty, (k_it & 1) ^ 1, s_abort, 802);
-                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 1);
-                    if (ok) mbar_arrive_expect_tx(my_k_full, kMla2KBytes);
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
+        // one thread: group g of the next tile is requested as soon as the MMAs that read group g of this tile are done
+        if (lane == 0) {
+            uint32_t q_it = 0, kc = 0, item_it = 0;
+            bool ok = true;
+            for (int item = pair; item < total_items && ok; item += num_pairs) {
+                WorkUnit u;
+                int h;
+                get_item(item, u, h);
+                ++item_it;
+                // Q may be replaced once the scores of the previous item's last tile are done
+                if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 801);
                 if (!ok) break;
-                blk = __shfl_sync(0xffffffffu, blk, 0);
-                slot_in = __shfl_sync(0xffffffffu, slot_in, 0);
-                if (lane < kMlaSlabs) tma_load_5d(sK + lane * 8192, &tm_k1, my_k_full, 0, slot_in, lane, 0, blk);
-                if (lane == 0) VPP_TR(3, j - u.kv_begin, 2);
-                if (lane == 0) VPP_TR1(2, j - u.kv_begin, 2);
-                ++k_it;
+                if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMla2QBytes);
+#pragma unroll 1
+                for (int s = 0; s < kMlaSlabs; ++s)
+                    tma2_load_4d(sQ + s * 8192, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, s, h);
+                ++q_it;
+                const int t_hi = tile_hi(u);
+                int blk_next = 0, slot_next = 0;
+                page_of(u, u.kv_begin * kTileN + static_cast<int>(rank) * 64, blk_next, slot_next);
+                for (int j = u.kv_begin; j < t_hi && ok; ++j) {
+                    const int blk = blk_next, slot_in = slot_next;
+                    if (j + 1 < t_hi) page_of(u, (j + 1) * kTileN + static_cast<int>(rank) * 64, blk_next, slot_next);
+                    const uint32_t par = (kc & 1) ^ 1;
+#pragma unroll 1
+                    for (int s = 0; s < kMlaSlabs; ++s) {
+                        const int g = s / kKG;
+                        if (s % kKG == 0) {
+                            if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, par, s_abort, 802);
+                            else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 802);
+                            if (!ok) break;
+                            VPP_TR(3, j - u.kv_begin, 4 + s);
+                            if (leader) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
+                        }
+                        tma2_load_5d(sK + s * 8192, &tm_k1, pair_k_full + 8 * g, 0, slot_in, s, 0, blk);
+                    }
+                    ++kc;
+                }
             }
         }
     } else if (warp == 6) {
         // ======================================= V producer =======================================
-        uint32_t v_it = 0, item_it = 0;
+        // chunk c = (key half hf, instr i) holds value columns 256 i + 128 rank .. + 127 of keys 64 hf .. 64 hf + 63.
+        // A tile that reaches past the end of the sequence is special: each CTA lands its part on a barrier of its
+        // own, zeroes the value rows of the keys that do not exist (0 * garbage must not reach O) and then arrives
+        // on bar_vfix, which the MMA thread waits on before it multiplies that tile.
+        uint32_t vc = 0, tails = 0;
         bool ok = true;
+        const uint32_t own_v_full = leader ? bar_v_full : bar_v_local;
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
             get_item(item, u, h);
-            ++item_it;
             const int t_hi = tile_hi(u);
+            int nb0 = 0, ns0 = 0, nb1 = 0, ns1 = 0;
+            if (lane == 0) {
+                page_of(u, u.kv_begin * kTileN, nb0, ns0);
+                page_of(u, u.kv_begin * kTileN + 64, nb1, ns1);
+            }
             for (int j = u.kv_begin; j < t_hi && ok; ++j) {
                 const int tile0 = j * kTileN;
-                int blk = 0, slot_in = 0;
-                if (lane < 2) page_of(u, tile0 + 64 * lane, blk, slot_in);   // lane hf looks up key half hf
+                const bool tail = tile0 + kTileN > u.kv_len;
                 if (lane == 0) {
-                    VPP_TR(3, j - u.kv_begin, 3);
-                    ok = mbar_wait(bar_v_empty, (v_it & 1) ^ 1, s_abort, 803);
-                    VPP_TR(3, j - u.kv_begin, 4);
-                    if (ok) mbar_arrive_expect_tx(my_v_full, kMla2VBytes);
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (ok) {
-                    // lane = hf*4 + i*2 + g copies value group g of instr i for key half hf: slab 4 i + 2 rank + g,
-                    // to [key half][instr][col group][64 keys][128 B]
-                    const int hf = (lane >> 2) & 1, ig = lane & 3;
-                    const int b2 = __shfl_sync(0xffffffffu, blk, hf), s2 = __shfl_sync(0xffffffffu, slot_in, hf);
-                    if (lane < 8)
-                        tma_load_5d(sV + lane * 8192, &tm_k1, my_v_full, 0, s2, 4 * (ig >> 1) + 2 * static_cast<int>(rank) + (ig & 1),
-                                    0, b2);
-                    if (lane == 0) VPP_TR(3, j - u.kv_begin, 5);
+                    const int b0 = nb0, s0 = ns0, b1 = nb1, s1 = ns1;
+                    if (j + 1 < t_hi) {
+                        page_of(u, tile0 + kTileN, nb0, ns0);
+                        page_of(u, tile0 + kTileN + 64, nb1, ns1);
+                    }
+                    const uint32_t par = (vc & 1) ^ 1;
+#pragma unroll 1
+                    for (int c = 0; c < kMla2VChunks; ++c) {
+                        const int g = c / kVG;
+                        if (c % kVG == 0) {
+                            if (g < kVGroups - 1) ok = mbar_wait(bar_v_empty + 8 * g, par, s_abort, 803);
+                            else if (vc > 0) ok = mbar_wait(bar_pv_done, (vc - 1) & 1, s_abort, 803);
+                            if (!ok) break;
+                            if (tail) mbar_arrive_expect_tx(own_v_full + 8 * g, kVG * kMla2VChunk);
+                            else if (leader) mbar_arrive_expect_tx(bar_v_full + 8 * g, 2 * kVG * kMla2VChunk);
+                        }
+                        const int hf = c >> 1, slab0 = 4 * (c & 1) + 2 * static_cast<int>(rank);
+                        const uint32_t dst = sV + c * kMla2VChunk;
+                        if (tail) {
+                            tma_load_5d(dst, &tm_k1, own_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
+                            tma_load_5d(dst + 8192, &tm_k1, own_v_full + 8 * g, 0, hf ? s1 : s0, slab0 + 1, 0, hf ? b1 : b0);
+                        } else {
+                            tma2_load_5d(dst, &tm_k1, pair_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
+                            tma2_load_5d(dst + 8192, &tm_k1, pair_v_full + 8 * g, 0, hf ? s1 : s0, slab0 + 1, 0, hf ? b1 : b0);
+                        }
+                    }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) break;
-                if (leader && tile0 + kTileN > u.kv_len) {
-                    // keys at or beyond kv_len do not exist: zero their value rows (0 * garbage must not reach O)
-                    if (lane == 0) ok = mbar_wait(bar_v_full, v_it & 1, s_abort, 804);
+                if (tail) {
+                    if (lane == 0) {
+                        for (int g = 0; g < kMla2VChunks / kVG && ok; ++g)
+                            ok = mbar_wait(own_v_full + 8 * g, leader ? (vc & 1) : (tails & 1), s_abort, 804);
+                    }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) break;
                     const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
-                    const uint4 z = make_uint4(0, 0, 0, 0);
-                    for (int r = first + lane; r < kTileN; r += 32) {
-                        const int hf = r >> 6, rr = r & 63;
-#pragma unroll
-                        for (int blk4 = 0; blk4 < 4; ++blk4) {  // 2 instr x 2 col groups
-                            uint4* a = reinterpret_cast<uint4*>(gen_base + kMla2QBytes + kMla2KBytes + hf * 32768 +
-                                                                blk4 * 8192 + rr * 128);
-#pragma unroll
-                            for (int c = 0; c < 8; ++c) a[c] = z;
-                        }
-                    }
+                    for (int c = 0; c < kMla2VChunks; ++c)
+                        if (first < (c >> 1) * 64 + 64) zero_v_rows(c, first);
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_vfix);
-                }
-                ++v_it;
-            }
-        }
-    } else if (warp == 1 && !leader) {
-        // ================================ relay (rank 1 only) ================================
-        uint32_t q_it = 0, kv_it = 0, item_it = 0;
-        bool ok = true;
-        for (int item = pair; item < total_items && ok; item += num_pairs) {
-            WorkUnit u;
-            int h;
-            get_item(item, u, h);
-            ++item_it;
-            if (lane == 0) {
-                ok = mbar_wait(bar_qk_local, q_it & 1, s_abort, 811);
-                if (ok) mbar_arrive_remote(bar_q_full, 0);
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            ++q_it;
-            const int t_hi = tile_hi(u);
-            for (int j = u.kv_begin; j < t_hi && ok; ++j) {
-                const int tile0 = j * kTileN;
-                if (lane == 0) {
-                    ok = mbar_wait(bar_qk_local + 8, kv_it & 1, s_abort, 812);
-                    VPP_TR1(2, j - u.kv_begin, 0);
-                    if (ok) mbar_arrive_remote(bar_k_full, 0);
-                    if (ok) ok = mbar_wait(bar_qk_local + 16, kv_it & 1, s_abort, 813);
-                    VPP_TR1(2, j - u.kv_begin, 1);
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) break;
-                if (tile0 + kTileN > u.kv_len) {
-                    const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
-                    const uint4 z = make_uint4(0, 0, 0, 0);
-                    for (int r = first + lane; r < kTileN; r += 32) {
-                        const int hf = r >> 6, rr = r & 63;
-#pragma unroll
-                        for (int blk4 = 0; blk4 < 4; ++blk4) {
-                            uint4* a = reinterpret_cast<uint4*>(gen_base + kMla2QBytes + kMla2KBytes + hf * 32768 +
-                                                                blk4 * 8192 + rr * 128);
-#pragma unroll
-                            for (int c = 0; c < 8; ++c) a[c] = z;
-                        }
+                    if (lane == 0) {
+                        if (leader) mbar_arrive(bar_vfix);
+                        else mbar_arrive_remote(bar_vfix, 0);
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
+                    ++tails;
                 }
-                if (lane == 0) mbar_arrive_remote(bar_v_full, 0);
-                ++kv_it;
+                ++vc;
             }
         }
     } else if (warp == 1 && leader && lane == 0) {
@@ -367,83 +399,99 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         const uint32_t q_lo = desc_lo_sw128(sQ, 16), k_lo = desc_lo_sw128(sK, 16), p_lo = desc_lo_sw128(sP, 16);
         const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
         const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
-        uint32_t q_it = 0, k_it = 0, v_it = 0, tc = 0, vfix_it = 0, item_it = 0;
-        auto issue_qk = [&](uint32_t tS) {
+        uint32_t q_it = 0, kc = 0, vc = 0, tc = 0, vfix_it = 0, item_it = 0;
+        bool ok = true;
+        // scores of K group g (kKG slabs) into tS; the group goes back to the producer when its MMAs are done and
+        // the last group's commit also tells the softmax warps that the scores are complete
+        auto qk_group = [&](uint32_t tS, int g, uint32_t bar_last) {
 #pragma unroll 1
-            for (int s = 0; s < kMlaSlabs; ++s)
+            for (int s = g * kKG; s < (g + 1) * kKG; ++s) {
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)
+                for (int kk = 0; kk < 4; ++kk) {
+#ifndef VPP_T2_NO_QK
                     mma2_ss_lh(tS, q_lo + ((s * 8192 + kk * 32) >> 4), k_lo + ((s * 8192 + kk * 32) >> 4), kHi, kIdescQK,
                                (s > 0 || kk > 0) ? 1u : 0u);
+#endif
+                }
+            }
+            tc_commit2(g < kKGroups - 1 ? bar_k_empty + 8 * g : bar_last, 3);
         };
-        bool ok = true;
+        // O += P V for V group g: chunk c = (key half c >> 1, output half c & 1)
+        auto pv_group = [&](int g, bool first_tile) {
+#pragma unroll 1
+            for (int c = g * kVG; c < (g + 1) * kVG; ++c) {
+                const uint32_t tO = (c & 1) ? tO1 : tO0;
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4) {
+#ifndef VPP_T2_NO_PV
+                    mma2_ss_lh(tO, p_lo + (((c >> 1) * 8192 + k4 * 32) >> 4), v_lo + ((c * kMla2VChunk + k4 * 2048) >> 4),
+                               kHi, kIdescPV, (!first_tile || c > 1 || k4 > 0) ? 1u : 0u);
+#endif
+                }
+            }
+            tc_commit2(g < kVGroups - 1 ? bar_v_empty + 8 * g : bar_pv_done, 3);
+        };
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
             get_item(item, u, h);
             const int n = tile_hi(u) - u.kv_begin;
             ++item_it;
-            ok = mbar_wait_cluster(bar_q_full, q_it & 1, s_abort, 821);
+            ok = mbar_wait(bar_q_full, q_it & 1, s_abort, 821);
             if (!ok) break;
             ++q_it;
-            ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 822);
+            for (int g = 0; g < kKGroups && ok; ++g) {
+                ok = mbar_wait(bar_k_full + 8 * g, kc & 1, s_abort, 822);
+                if (!ok) break;
+                tc_fence_after();
+                qk_group(tmem_base + (tc & 1) * 64, g, bar_s_full + 8 * (tc & 1));
+            }
             if (!ok) break;
-            ++k_it;
-            tc_fence_after();
-            issue_qk(tmem_base + (tc & 1) * 64);
-            tc_commit2(bar_k_empty, 3);
-            tc_commit2(bar_s_full + 8 * (tc & 1), 3);
-            if (n == 1) tc_commit2(bar_q_empty, 3);
+            ++kc;
             for (int jj = 0; jj < n; ++jj) {
                 const int tile0 = (u.kv_begin + jj) * kTileN;
                 const uint32_t b = tc & 1;
+                const bool tail = tile0 + kTileN > u.kv_len;
                 VPP_TR(0, jj, 0);
-                // Scores of the next tile first if its keys are already here (they overlap this tile's softmax);
-                // otherwise P V of this tile goes first so that the tensor core is not idle while the keys arrive.
-                auto next_scores = [&]() {
-                    ++k_it;
-                    tc_fence_after();
-                    VPP_TR(0, jj, 1);
-                    issue_qk(tmem_base + (b ^ 1) * 64);
-                    VPP_TR(0, jj, 2);
-                    tc_commit2(bar_k_empty, 3);
-                    tc_commit2(bar_s_full + 8 * (b ^ 1), 3);
-                    if (jj + 2 == n) tc_commit2(bar_q_empty, 3);
-                };
-                bool scores_done = jj + 1 >= n;
-                if (!scores_done && mbar_try_wait_cluster(bar_k_full, k_it & 1)) {
-                    next_scores();
-                    scores_done = true;
+                // Two streams of work: the scores of tile jj + 1 (they overlap this tile's softmax) and P V of this
+                // tile.  Whichever has its operands in shared memory is issued next, scores first.
+                const int nq = jj + 1 < n ? kKGroups : 0;
+                int qg = 0, pg = 0, spins = 0;
+                bool p_ready = false;
+                long long t0 = 0;
+                while (qg < nq || pg < kVGroups) {
+                    if (qg < nq && mbar_try_wait(bar_k_full + 8 * qg, kc & 1)) {
+                        tc_fence_after();
+                        VPP_TR(2, jj, qg);
+                        qk_group(tmem_base + (b ^ 1) * 64, qg, bar_s_full + 8 * (b ^ 1));
+                        ++qg;
+                        continue;
+                    }
+                    if (!p_ready)
+                        p_ready = mbar_try_wait_cluster(bar_p_full + 8 * b, (tc >> 1) & 1) &&
+                                  (!tail || mbar_try_wait_cluster(bar_vfix, vfix_it & 1));
+                    if (p_ready && mbar_try_wait(bar_v_full + 8 * pg, vc & 1)) {
+                        tc_fence_after();
+                        VPP_TR(3, jj, pg);
+                        pv_group(pg, jj == 0);
+                        ++pg;
+                        continue;
+                    }
+                    if ((++spins & 63) == 0) {
+                        if (t0 == 0) t0 = clock64();
+                        if (*s_abort != 0) ok = false;
+                        else if (clock64() - t0 > kWaitLimitCycles) {
+                            atomicCAS(const_cast<int*>(s_abort), 0, 826);
+                            ok = false;
+                        }
+                        if (!ok) break;
+                    }
                 }
-                ok = mbar_wait_cluster(bar_v_full, v_it & 1, s_abort, 824);
                 if (!ok) break;
-                ++v_it;
-                VPP_TR(0, jj, 3);
-                if (tile0 + kTileN > u.kv_len) {
-                    ok = mbar_wait(bar_vfix, vfix_it & 1, s_abort, 825);
-                    if (!ok) break;
-                    ++vfix_it;
-                }
-                ok = mbar_wait_cluster(bar_p_full + 8 * b, (tc >> 1) & 1, s_abort, 826);
-                if (!ok) break;
-                tc_fence_after();
-                VPP_TR(0, jj, 4);
-#pragma unroll
-                for (int i = 0; i < 2; ++i)
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        mma2_ss_lh(i == 0 ? tO0 : tO1, p_lo + (((kk >> 2) * 8192 + (kk & 3) * 32) >> 4),
-                                   v_lo + ((((kk >> 2) * 2 + i) * 16384 + (kk & 3) * 2048) >> 4), kHi, kIdescPV,
-                                   (jj > 0 || kk > 0) ? 1u : 0u);
-                tc_commit2(bar_v_empty, 3);
-                tc_commit2(bar_p_empty, 3);
                 VPP_TR(0, jj, 5);
-                if (jj + 1 == n) tc_commit2(bar_o_full, 3);
-                if (!scores_done) {
-                    ok = mbar_wait_cluster(bar_k_full, k_it & 1, s_abort, 823);
-                    if (!ok) break;
-                    next_scores();
-                }
+                if (nq) ++kc;
+                if (tail) ++vfix_it;
+                ++vc;
                 ++tc;
             }
         }
@@ -455,7 +503,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const uint32_t tO0 = tmem_base + 128 + lane_off, tO1 = tmem_base + 256 + lane_off;
         uint8_t* p_row = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + half * 8192 + row * 128;
-        uint32_t tc = 0, o_it = 0, x_it = 0, pe_it = 0, item_it = 0;
+        uint32_t tc = 0, x_it = 0, item_it = 0;
         const float sc = p.scale_log2e;
         auto exchange = [&](float mine, float& theirs) -> bool {
             float* buf = xch + (x_it & 1) * 128;
@@ -510,11 +558,17 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 if (l128 == 0) VPP_TR(1, j - u.kv_begin, 2);
                 const float m_new = fmaxf(fmaxf(mxa, mxb) * sc, m_ref);
                 const bool grow = (m_new - m_ref > 8.f) || (m_ref == -INFINITY && m_new != -INFINITY);
+                bool p_free = false;
                 if (__any_sync(0xffffffffu, grow)) {
                     const float alpha = grow ? ex2(m_ref - m_new) : 1.f;
                     if (grow) m_ref = m_new;
                     l_run *= alpha;
                     if (j > u.kv_begin) {
+                        // O is rescaled in place: P V of the previous tile (issued after this tile's scores) must be done
+                        ok = mbar_wait(bar_pv_done, (tc - 1) & 1, s_abort, 835);
+                        if (!ok) break;
+                        p_free = true;
+                        tc_fence_after();
                         uint32_t o[32];
 #pragma unroll 1
                         for (int c = 0; c < 8; ++c) {
@@ -542,10 +596,9 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 l_run += sum0 + sum1;
                 if (l128 == 0) VPP_TR(1, j - u.kv_begin, 3);
                 // P of the previous tile must have been consumed before its shared-memory rows are overwritten
-                if (tc > 0) {
-                    ok = mbar_wait(bar_p_empty, pe_it & 1, s_abort, 833);
+                if (tc > 0 && !p_free) {
+                    ok = mbar_wait(bar_pv_done, (tc - 1) & 1, s_abort, 833);
                     if (!ok) break;
-                    ++pe_it;
                 }
 #pragma unroll
                 for (int c = 0; c < 8; ++c)  // K-major 128B-swizzled row: 16-byte chunk index XOR (row & 7)
@@ -567,9 +620,8 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             ok = exchange(l_run, l_other);
             if (!ok) break;
             const float l_tot = l_run + l_other;
-            ok = mbar_wait(bar_o_full, o_it & 1, s_abort, 834);
+            ok = mbar_wait(bar_pv_done, (tc - 1) & 1, s_abort, 834);  // P V of the item's last tile
             if (!ok) break;
-            ++o_it;
             tc_fence_after();
             const float inv_l = 1.f / l_tot;
             const bool live = my_row < u.rows;
