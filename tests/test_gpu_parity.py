@@ -73,6 +73,36 @@ def test_mla_adversarial_shapes(case, splits):
     print(s)
 
 
+def _ramp_scores(prob, step):
+    """Make the scores grow along the sequence: key p gets its last feature = p * step (for absorbed MLA that
+    feature is not part of the values), every query the same feature = 1, so the
+    running row maximum rises by more than the rescale threshold at every KV tile (the lazy rescale of O fires
+    on each tile instead of almost never)."""
+    bs = prob.k_cache.shape[1]
+    for r in range(len(prob.prefix_len)):
+        n = int(prob.prefix_len[r] + prob.chunk_len[r])
+        pos = torch.arange(n)
+        if prob.block_table is None:
+            prob.k_cache[r, pos, :, -1] = (pos.float() * step).to(prob.k_cache.dtype)[:, None]
+        else:
+            blk = prob.block_table[r, pos // bs].long()
+            prob.k_cache[blk, pos % bs, :, -1] = (pos.float() * step).to(prob.k_cache.dtype)[:, None]
+    prob.q[:, :, -1] = 1.0
+
+
+@pytest.mark.parametrize("family", ["gqa", "mla"])
+@pytest.mark.parametrize("splits", [0, 2])
+def test_running_maximum_grows_every_tile(family, splits):
+    if family == "gqa":
+        prob = W.make_problem(2200, [2000, 700], [300, 129], 4, 2, 128, 128, block_size=16, std=0.5)
+    else:
+        prob = W.make_problem(2201, [2000, 700], [300, 129], 4, 1, 576, 512, block_size=64, std=0.5,
+                              scale=1.0 / 192 ** 0.5, v_aliases_k=True)
+    _ramp_scores(prob, 1.0)   # scale * 128 keys * 1.0 is about 9-11 nats per tile, well above the 2^8 threshold
+    s, _ = full_check(prob, num_kv_splits=splits, label="%s ramp S=%d" % (family, splits))
+    print(s)
+
+
 def test_mla_requires_aliased_values():
     prob = W.make_problem(2100, [10], [20], 2, 1, 576, 512, block_size=16, std=0.5, v_aliases_k=True).to("cuda")
     runner = api.ChunkAttn(prob)
