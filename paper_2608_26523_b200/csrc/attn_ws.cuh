@@ -466,11 +466,11 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             if (hh * 64 + i > lim) s[hh * 64 + i] = 0xff800000u;  // -inf
                     }
 #pragma unroll
-                    for (int i = 0; i < 64; i += 8)
+                    for (int i = 0; i < 64; i += 16)
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            const float v = __uint_as_float(s[hh * 64 + i + k]);
-                            mx[k] = (hh == 0 && i == 0) ? v : fmaxf(mx[k], v);
+                            const float v0 = __uint_as_float(s[hh * 64 + i + k]), v1 = __uint_as_float(s[hh * 64 + i + 8 + k]);
+                            mx[k] = (hh == 0 && i == 0) ? fmaxf(v0, v1) : fmax3(mx[k], v0, v1);
                         }
                 }
                 const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),

@@ -267,6 +267,12 @@ __device__ __forceinline__ float ex2_poly(float x) {
     p = fmaf(p, f, 1.0000026226043701f);
     return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xf) << 23));
 }
+// three-input maximum (one instruction on sm_100)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
