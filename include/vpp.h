@@ -187,6 +187,49 @@ size_t vpp_static_scratch_bytes(void);
 /* Thread-local detail of the last failure of vpp_chunk_attn_fwd_static on this host thread. */
 const char *vpp_static_last_error(void);
 
+/*
+ * Paged KV-cache append: the step before vpp_chunk_attn_fwd in a chunked prefill (the paper's
+ * "Chunked Prefill Pipeline Parallelism" section: every chunk's keys and values join the cache that
+ * the later chunks attend to).  Row i of request r (0 <= i < chunk_len[r]) is written to position
+ * prefix_len[r] + i of that request: block block_table[r][pos / block_size], slot pos % block_size
+ * (block_table NULL: request r is block r and slot = pos).  Pure data movement, bit-exact.
+ *
+ * k_new        bf16 [total_q, num_kv_heads, head_dim_qk], dense, packed request-major like q. 16-byte aligned.
+ * v_new        bf16 [total_q, num_kv_heads, head_dim_v], or NULL when the values are the leading features of
+ *              the keys (v_cache aliases k_cache: absorbed MLA) -- then only the keys are written.
+ * k_cache, v_cache, strides, block_table, prefix_len, chunk_len, num_reqs, max_blocks_per_req, block_size,
+ * num_blocks, total_q: as in vpp_chunk_attn_args (the caches are written here, not read).  For a contiguous
+ *              cache (block_table NULL) max_seq_len is the number of positions each request's region holds.
+ * status       optional device int32, zeroed by the call.  VPP_DEV_BAD_LENGTHS: a negative length, a request
+ *              that would outgrow its pages, or sum(chunk_len) != total_q -- nothing is written.
+ *              VPP_DEV_BAD_BLOCK: a needed block_table entry outside [0, num_blocks) -- that row is skipped.
+ * head dims must be multiples of 8 elements, num_reqs at most 8192.  Rows of one call never overlap, so the
+ * result does not depend on scheduling.  Returns after enqueueing one kernel on `stream`.
+ */
+typedef struct {
+    const void *k_new;
+    const void *v_new;
+    void *k_cache;
+    void *v_cache;
+    int64_t k_block_stride, k_token_stride, k_head_stride;
+    int64_t v_block_stride, v_token_stride, v_head_stride;
+    const int32_t *block_table;
+    const int32_t *prefix_len;
+    const int32_t *chunk_len;
+    int32_t num_reqs;
+    int32_t max_blocks_per_req;
+    int32_t block_size;
+    int32_t num_blocks;
+    int32_t total_q;
+    int32_t max_seq_len;
+    int32_t num_kv_heads;
+    int32_t head_dim_qk;
+    int32_t head_dim_v;
+    int32_t *status;
+} vpp_kv_append_args;
+
+vpp_status vpp_kv_append(const vpp_kv_append_args *args, vpp_stream_t stream);
+
 /* Static description of a status code. */
 const char *vpp_status_string(vpp_status s);
 

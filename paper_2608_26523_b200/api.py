@@ -20,7 +20,7 @@ VPP_ERR_TIMEOUT = -5
 
 EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_status_string",
            "vpp_last_error", "vpp_last_launch_count", "vpp_chunk_attn_fwd_static", "vpp_static_scratch_bytes",
-           "vpp_static_last_error"]
+           "vpp_static_last_error", "vpp_kv_append"]
 
 
 class VppError(RuntimeError):
@@ -41,6 +41,19 @@ class ChunkAttnArgs(ctypes.Structure):
         ("head_dim_v", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("num_kv_splits", ctypes.c_int32),
         ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+    ]
+
+
+class KvAppendArgs(ctypes.Structure):
+    _fields_ = [
+        ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p), ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+        ("k_block_stride", ctypes.c_int64), ("k_token_stride", ctypes.c_int64), ("k_head_stride", ctypes.c_int64),
+        ("v_block_stride", ctypes.c_int64), ("v_token_stride", ctypes.c_int64), ("v_head_stride", ctypes.c_int64),
+        ("block_table", ctypes.c_void_p), ("prefix_len", ctypes.c_void_p), ("chunk_len", ctypes.c_void_p),
+        ("num_reqs", ctypes.c_int32), ("max_blocks_per_req", ctypes.c_int32), ("block_size", ctypes.c_int32),
+        ("num_blocks", ctypes.c_int32), ("total_q", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32), ("head_dim_qk", ctypes.c_int32), ("head_dim_v", ctypes.c_int32),
+        ("status", ctypes.c_void_p),
     ]
 
 
@@ -70,6 +83,8 @@ def load_library():
         lib.vpp_chunk_attn_fwd_static.argtypes = [ctypes.POINTER(ChunkAttnArgs), ctypes.c_void_p]
         lib.vpp_static_scratch_bytes.restype = ctypes.c_size_t
         lib.vpp_static_last_error.restype = ctypes.c_char_p
+        lib.vpp_kv_append.restype = ctypes.c_int
+        lib.vpp_kv_append.argtypes = [ctypes.POINTER(KvAppendArgs), ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -154,6 +169,34 @@ def vpp_lse_merge(o_parts, lse_parts, out, lse=None, stream=None):
         stream = torch.cuda.current_stream().cuda_stream
     _check(load_library().vpp_lse_merge(_ptr(o_parts), _ptr(lse_parts), S, T, Hq, Dv, _ptr(out), _ptr(lse),
                                         ctypes.c_void_p(stream)))
+
+
+def vpp_kv_append(k_new, v_new, k_cache, v_cache, block_table, prefix_len, chunk_len, block_size, max_seq_len,
+                  status=None, stream=None, total_q=None):
+    """Write the chunk's new K/V rows into the (paged) cache: row i of request r goes to position prefix_len[r] + i.
+
+    k_new [T, Hkv, Dqk] bf16, v_new [T, Hkv, Dv] bf16 or None when v_cache is a view of k_cache (absorbed MLA);
+    caches [num_blocks, block_size, Hkv, D] with a contiguous last dim; block_table int32 [R, max_blocks] or None."""
+    a = KvAppendArgs()
+    a.k_new, a.v_new, a.k_cache, a.v_cache = _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache)
+    ks = k_cache.stride()
+    vs = v_cache.stride() if v_cache is not None else (0, 0, 0, 1)
+    assert ks[3] == 1 and vs[3] == 1 and k_new.is_contiguous() and (v_new is None or v_new.is_contiguous())
+    a.k_block_stride, a.k_token_stride, a.k_head_stride = ks[0], ks[1], ks[2]
+    a.v_block_stride, a.v_token_stride, a.v_head_stride = vs[0], vs[1], vs[2]
+    a.block_table, a.prefix_len, a.chunk_len = _ptr(block_table), _ptr(prefix_len), _ptr(chunk_len)
+    a.num_reqs = prefix_len.numel()
+    a.max_blocks_per_req = 0 if block_table is None else block_table.shape[1]
+    a.block_size = int(block_size)
+    a.num_blocks = k_cache.shape[0]
+    a.total_q = k_new.shape[0] if total_q is None else int(total_q)
+    a.max_seq_len = int(max_seq_len)
+    a.num_kv_heads, a.head_dim_qk = k_new.shape[1], k_new.shape[2]
+    a.head_dim_v = v_new.shape[2] if v_new is not None else (v_cache.shape[3] if v_cache is not None else k_new.shape[2])
+    a.status = _ptr(status)
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_kv_append(ctypes.byref(a), ctypes.c_void_p(stream)))
 
 
 def vpp_last_launch_count():

@@ -16,6 +16,7 @@
 #include "attn_mla2.cuh"
 #include "attn_ws.cuh"
 #include "common.cuh"
+#include "kv_append.cuh"
 #include "merge.cuh"
 #include "prep.cuh"
 
@@ -454,6 +455,71 @@ vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t n
         lse);
     cudaError_t ce = cudaGetLastError();
     if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "merge launch: %s", cudaGetErrorString(ce));
+    return VPP_OK;
+}
+
+vpp_status vpp_kv_append(const vpp_kv_append_args* a, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    if (!a) return fail(VPP_ERR_INVALID_ARG, "args is null");
+    if (a->num_reqs < 0 || a->total_q < 0 || a->num_kv_heads <= 0 || a->head_dim_qk <= 0 || a->head_dim_v <= 0)
+        return fail(VPP_ERR_INVALID_ARG, "num_reqs, total_q >= 0 and num_kv_heads, head dims > 0 required");
+    if (a->head_dim_qk % 8 || a->head_dim_v % 8) return fail(VPP_ERR_UNSUPPORTED, "head dims must be multiples of 8");
+    if (a->num_reqs > vpp::kAppendMaxReqs) return fail(VPP_ERR_UNSUPPORTED, "at most %d requests", vpp::kAppendMaxReqs);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (a->status && cudaMemsetAsync(a->status, 0, sizeof(int32_t), stream) != cudaSuccess)
+        return fail(VPP_ERR_CUDA, "memset status: %s", cudaGetErrorString(cudaGetLastError()));
+    if (a->total_q == 0 || a->num_reqs == 0) return VPP_OK;
+    if (!a->k_new || !a->k_cache || !a->prefix_len || !a->chunk_len)
+        return fail(VPP_ERR_INVALID_ARG, "k_new, k_cache, prefix_len and chunk_len must be non-null");
+    if (a->v_new && !a->v_cache) return fail(VPP_ERR_INVALID_ARG, "v_new given without v_cache");
+    int shift = 0;
+    long long capacity = a->max_seq_len;
+    if (a->block_table) {
+        if (a->block_size < 1 || (a->block_size & (a->block_size - 1)))
+            return fail(VPP_ERR_UNSUPPORTED, "block_size must be a power of two");
+        if (a->max_blocks_per_req <= 0 || a->num_blocks <= 0)
+            return fail(VPP_ERR_INVALID_ARG, "max_blocks_per_req and num_blocks must be > 0 with a block table");
+        while ((1 << shift) < a->block_size) ++shift;
+        capacity = static_cast<long long>(a->max_blocks_per_req) * a->block_size;
+    } else if (a->max_seq_len <= 0) {
+        return fail(VPP_ERR_INVALID_ARG, "max_seq_len must be > 0 for a contiguous cache");
+    }
+    const int64_t strides[6] = {a->k_block_stride, a->k_token_stride, a->k_head_stride,
+                                a->v_block_stride, a->v_token_stride, a->v_head_stride};
+    for (int i = 0; i < (a->v_new ? 6 : 3); ++i)
+        if (strides[i] < 0 || strides[i] % 8) return fail(VPP_ERR_INVALID_ARG, "strides must be non-negative multiples of 8 elements");
+    uintptr_t al = reinterpret_cast<uintptr_t>(a->k_new) | reinterpret_cast<uintptr_t>(a->k_cache);
+    if (a->v_new) al |= reinterpret_cast<uintptr_t>(a->v_new) | reinterpret_cast<uintptr_t>(a->v_cache);
+    if (al & 15u) return fail(VPP_ERR_INVALID_ARG, "k_new, v_new and the caches must be 16-byte aligned");
+
+    vpp::AppendParams p{};
+    p.k_new = static_cast<const uint4*>(a->k_new);
+    p.v_new = static_cast<const uint4*>(a->v_new);
+    p.k_cache = static_cast<uint8_t*>(a->k_cache);
+    p.v_cache = static_cast<uint8_t*>(a->v_cache);
+    p.k_block_stride = a->k_block_stride * 2; p.k_token_stride = a->k_token_stride * 2; p.k_head_stride = a->k_head_stride * 2;
+    p.v_block_stride = a->v_block_stride * 2; p.v_token_stride = a->v_token_stride * 2; p.v_head_stride = a->v_head_stride * 2;
+    p.block_table = a->block_table;
+    p.prefix_len = a->prefix_len;
+    p.chunk_len = a->chunk_len;
+    p.num_reqs = a->num_reqs;
+    p.max_blocks_per_req = a->max_blocks_per_req;
+    p.block_shift = shift;
+    p.num_blocks = a->num_blocks;
+    p.capacity = capacity;
+    p.total_q = a->total_q;
+    p.num_kv_heads = a->num_kv_heads;
+    p.k_vecs = a->head_dim_qk / 8;
+    p.v_vecs = a->v_new ? a->head_dim_v / 8 : 0;
+    p.status = a->status;
+    const int rows_per_block = vpp::kAppendThreads / 32;
+    long long blocks = (static_cast<long long>(a->total_q) + rows_per_block - 1) / rows_per_block;
+    const long long cap = 16ll * sm_count_or_default();
+    if (blocks > cap) blocks = cap;
+    const size_t smem = sizeof(int32_t) * (static_cast<size_t>(a->num_reqs) + 1);
+    vpp::kv_append_kernel<<<static_cast<unsigned>(blocks), vpp::kAppendThreads, smem, stream>>>(p);
+    cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "append launch: %s", cudaGetErrorString(ce));
     return VPP_OK;
 }
 

@@ -74,6 +74,20 @@ def test_layout_of_args_struct_matches_header(tmp_path):
                  A.status.offset]
 
 
+def test_layout_of_append_args_matches_header(tmp_path):
+    import subprocess
+    src = tmp_path / "layout2.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "vpp.h"\n'
+                   'int main(void){printf("%zu %zu %zu %zu %zu\\n", sizeof(vpp_kv_append_args),'
+                   'offsetof(vpp_kv_append_args, k_cache), offsetof(vpp_kv_append_args, block_table),'
+                   'offsetof(vpp_kv_append_args, num_reqs), offsetof(vpp_kv_append_args, status));return 0;}\n')
+    exe = tmp_path / "layout2"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)])
+    c = [int(x) for x in subprocess.check_output([str(exe)]).split()]
+    A = api.KvAppendArgs
+    assert c == [ctypes.sizeof(A), A.k_cache.offset, A.block_table.offset, A.num_reqs.offset, A.status.offset]
+
+
 @pytest.mark.parametrize("mutate,status", [
     (lambda a: setattr(a, "head_dim_qk", 96), api.VPP_ERR_UNSUPPORTED),
     (lambda a: setattr(a, "num_kv_heads", 3), api.VPP_ERR_INVALID_ARG),
