@@ -132,13 +132,75 @@ def oracle_sample_rate(prob_cpu, target_seconds, rng):
     return fl, dt, n, threads
 
 
+def bench_append(args):
+    """The KV-cache append kernel (the step before attention) against the HBM roofline: bytes read + written per call
+    divided by the CUDA-event time.  Small chunks cycle through enough distinct buffers to exceed the L2."""
+    import torch
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    gen = torch.Generator(device="cpu").manual_seed(W.BASE_SEED + 77)
+    cases = [("cfg2 chunk: T=8192 Hkv=4 d=128, 128-token pages", 8192, 4, 128, 128, 128, False),
+             ("cfg4 chunk: T=16384 Hkv=8 d=128, 128-token pages", 16384, 8, 128, 128, 128, False),
+             ("cfg3 chunk: T=8192 latent 576 (values alias keys), 64-token pages", 8192, 1, 576, 512, 64, True),
+             ("large: T=262144 Hkv=8 d=128, 128-token pages", 262144, 8, 128, 128, 128, False)]
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    for desc, T, hkv, dqk, dv, bs, alias in cases:
+        bytes_call = T * hkv * (dqk + (0 if alias else dv)) * 2 * 2           # read + written
+        sets = max(1, int(math.ceil(400e6 / bytes_call)))                       # distinct buffers > 126 MB L2
+        nblk = T // bs
+        k_new = [torch.randn(T, hkv, dqk, generator=gen).to(torch.bfloat16).to(dev) for _ in range(min(sets, 4))]
+        v_new = None if alias else [x[..., :dv].contiguous() for x in k_new]
+        k_cache = [torch.zeros(nblk, bs, hkv, dqk, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        v_cache = [kc[..., :dv] for kc in k_cache] if alias else [torch.zeros_like(kc) for kc in k_cache]
+        bt = torch.randperm(nblk, generator=gen).to(torch.int32).view(1, nblk).to(dev)
+        pre = torch.zeros(1, dtype=torch.int32, device=dev)
+        cl = torch.full((1,), T, dtype=torch.int32, device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        def call(i):
+            api.vpp_kv_append(k_new[i % len(k_new)], None if alias else v_new[i % len(k_new)], k_cache[i % sets],
+                              v_cache[i % sets], bt, pre, cl, bs, T, status=status, stream=stream.cuda_stream)
+        n = max(args.steps, 5) * max(1, sets // 4)
+        with torch.cuda.stream(stream):
+            for i in range(max(args.warmup, 3)):
+                call(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(n):
+                call(i)
+            e1.record(stream)
+        e1.synchronize()
+        assert int(status.item()) == 0
+        ms = e0.elapsed_time(e1) / n
+        rows.append({"case": desc, "us": round(ms * 1e3, 2), "GB/s": round(bytes_call / ms / 1e6, 1),
+                     "frac_of_hbm_peak": round(bytes_call / ms / 1e6 / peaks["hbm_gbs"], 4), "bytes": bytes_call,
+                     "launches_timed": n})
+        del k_new, v_new, k_cache, v_cache
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[-1]
+    print(json.dumps({"metric": "kv-append GB/s (read + written) vs HBM peak (1 B200)", "value": top["GB/s"], "unit": "GB/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "dtype": "bf16 (bytes moved)",
+                      "data": "synthetic", "config": {"workload": "kv-append; " + top["case"], "l2": "distinct buffers of 400 MB or more per case"},
+                      "cases": rows, "vs_baseline": None,
+                      "roofline": {"bound": "hbm", "achieved": top["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": top["frac_of_hbm_peak"], "traffic": None,
+                                   "peak_source": "%s (copy bandwidth)" % peaks["_source"], "kernel": "kv_append_kernel, " + top["case"]},
+                      "gpu_launches": sum(r["launches_timed"] for r in rows), "clocks": clocks}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -147,6 +209,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
+    if args.workload == "append":
+        return bench_append(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,
