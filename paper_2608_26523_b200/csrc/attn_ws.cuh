@@ -265,9 +265,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr uint32_t kHi = desc_hi_sw128(1024);
             const uint32_t q_lo0 = desc_lo_sw128(sQ, 16), q_lo1 = desc_lo_sw128(sQ + kTileBytes, 16);
             auto issue_qk = [&](uint32_t tS, uint32_t q_lo, uint32_t k_stage) {
-#ifdef VPP_T_NO_QK
-                return;
-#endif
                 const uint32_t k_lo = desc_lo_sw128(k_stage, 16);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
@@ -276,21 +273,10 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             };
             auto issue_pv = [&](uint32_t tO, uint32_t tP, uint32_t v_stage, bool first, int k0, int k1) {
-#ifdef VPP_T_NO_PV
-                return;
-#endif
                 const uint32_t v_lo = desc_lo_sw128(v_stage, kSlabBytes);
 #pragma unroll
                 for (int k = k0; k < k1; ++k) {
-#if defined(VPP_T_PV_KMAJOR)   // timing experiment: wrong results
-                    const uint32_t koff = ((k >> 2) * kSlabBytes + (k & 3) * 32) >> 4;
-                    mma_ts_lh(tO, tP + k * 8, desc_lo_sw128(v_stage, 16) + koff, kHi, kIdescQK, (!first || k > 0) ? 1u : 0u);
-#elif defined(VPP_T_PV_SS)     // timing experiment: wrong results
-                    const uint32_t koff = ((k >> 2) * kSlabBytes + (k & 3) * 32) >> 4;
-                    mma_ss_lh(tO, q_lo0 + koff, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
-#else
                     mma_ts_lh(tO, tP + k * 8, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
-#endif
                 }
             };
             while (true) {
@@ -502,16 +488,11 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     uint32_t pk[16];
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
-#ifdef VPP_EXP_FAKE  // timing experiment only: results are wrong
-                        const float p0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
-                        const float p1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
-#else
                         const float x0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
                         const float x1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
                         // optionally every kEmuEvery-th exponential runs on the FMA pipe instead of the SFU
                         const float p0 = (kEmuEvery > 0 && (i % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x0) : ex2(x0);
                         const float p1 = (kEmuEvery > 0 && ((i + 1) % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x1) : ex2(x1);
-#endif
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);

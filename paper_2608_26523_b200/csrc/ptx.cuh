@@ -59,9 +59,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     int spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-#ifdef VPP_WAIT_SLEEP
-        __nanosleep(VPP_WAIT_SLEEP);
-#endif
         if ((++spins & 63) == 0) {
             if (*abort_flag != 0) return false;
             if (clock64() - t0 > kWaitLimitCycles) {
