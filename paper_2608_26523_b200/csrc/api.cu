@@ -305,8 +305,16 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_v, a->v_cache, 4, d, s, b)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(v) failed");
     }
 
-    CUtensorMap tm_q2, tm_k2, tm_v2;
+    CUtensorMap tm_q2, tm_k2, tm_v2, tm_qh;
     if (fam == Family::kGqa128) {
+        // a single-token ("packed") work item takes the G q-heads of one kv-head as the rows of its Q tile
+        const int G = a->num_q_heads / a->num_kv_heads;
+        const uint64_t dh[3] = {static_cast<uint64_t>(a->head_dim_qk), static_cast<uint64_t>(a->num_q_heads),
+                                static_cast<uint64_t>(a->total_q)};
+        const uint64_t sh[2] = {static_cast<uint64_t>(a->head_dim_qk) * 2,
+                                static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2};
+        const uint32_t bh[3] = {64, static_cast<uint32_t>(G < vpp::kTileM ? G : vpp::kTileM), 1};
+        if (!make_tmap(&tm_qh, a->q, 3, dh, sh, bh)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(q heads) failed");
         // the 128 features viewed as (64, 2): a box holds both 64-column slabs of a tile
         const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), 2, static_cast<uint64_t>(a->num_q_heads)};
         const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
@@ -410,7 +418,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     } else if (use_ws_kernel(a)) {
         auto kern = vpp::attn128_ws_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, ap, box_rows);
+        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, tm_qh, ap, box_rows);
     } else {
         auto kern = vpp::attn128_simple_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);

@@ -13,6 +13,9 @@
 //               from tensor memory, P_0 written back to tensor memory as bf16 over S_0.
 //   warps 8-11  the same for tile 1.
 // While one group works on its S tile the tensor core runs the other tile's MMAs.
+// A work unit of a single query token (a decode step batched with prefill chunks, or the one-row tail of a chunk) is
+// run "packed": the G q-heads that share a kv-head become the rows of tile 0, so its K/V is streamed once per
+// kv-head instead of once per pair of q-heads; tile 1 and its softmax group sit the item out.
 // Tensor memory: S_0 | S_1 | O_0 | O_1, 128 fp32 columns each (all 512 columns).
 //
 // The math per row is the paper's Eq. 1 with the causal rule, evaluated KV tile by KV tile with a
@@ -45,9 +48,10 @@ constexpr int kEmuEvery = VPP_EMU_EVERY;      // 0: all exponentials on the SFU 
 
 struct WsItem {
     WorkUnit u;
-    int32_t h0;     // first of the two q-heads
-    int32_t valid;  // 0: no more work
-    int32_t pad[2];
+    int32_t h0;      // first of the two q-heads (packed item: first head of the kv-head's group)
+    int32_t valid;   // 0: no more work
+    int32_t packed;  // 1: single-token item, the rows of tile 0 are the G q-heads of one kv-head; tile 1 is unused
+    int32_t pad;
 };
 
 
@@ -55,7 +59,8 @@ __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_q2,
                   const __grid_constant__ CUtensorMap tm_k2, const __grid_constant__ CUtensorMap tm_v2,
-                  const AttnParams p, const int kv_box_rows) {
+                  const __grid_constant__ CUtensorMap tm_qh, const AttnParams p, const int kv_box_rows) {
+    // tm_qh: the q tensor with a box of (64 features, G heads, 1 token): the rows of a packed item's Q tile
     // tm_q2 / tm_k2 / tm_v2 are views of the same tensors with the 128 features split into (64, 2): one box
     // of them brings both 64-column slabs of a 128-row tile, i.e. a whole tile per copy instruction.  Issuing a
     // copy costs the producer thread several hundred cycles, so fewer, larger copies matter.  tm_k / tm_v
@@ -111,6 +116,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         prefetch_tmap(&tm_q2);
         prefetch_tmap(&tm_k2);
         prefetch_tmap(&tm_v2);
+        prefetch_tmap(&tm_qh);
     }
     __syncthreads();
     if (warp == 2) {
@@ -135,23 +141,28 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (lane == 0) item = atomicAdd(&p.header->counter, 1);
                 item = __shfl_sync(0xffffffffu, item, 0);
                 const bool have = item < total_items;
-                const uint32_t slot = item_it & 1;
-                bool ok = true;
-                if (lane == 0) ok = mbar_wait(bar_item_empty + 8 * slot, ((item_it >> 1) & 1) ^ 1, s_abort, 201);
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (!ok) break;
                 WorkUnit u{};
                 int h0 = 0;
+                bool packed = false;
                 if (have) {
                     int ui, hp;
                     decode_item(item, num_units, p.num_q_heads / 2, G / 2, ui, hp);
                     u = p.units[ui];
                     h0 = 2 * hp;
+                    packed = u.rows == 1 && G <= kTileM;
+                    // a packed unit is served by the first head slot of each kv-head; its other slots have nothing to do
+                    if (packed && h0 % G != 0) continue;
                 }
+                const uint32_t slot = item_it & 1;
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(bar_item_empty + 8 * slot, ((item_it >> 1) & 1) ^ 1, s_abort, 201);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
                 if (lane == 0) {
                     ring[slot].u = u;
                     ring[slot].h0 = h0;
                     ring[slot].valid = have ? 1 : 0;
+                    ring[slot].packed = packed ? 1 : 0;
                     mbar_arrive(bar_item_full + 8 * slot);
                 }
                 ++item_it;
@@ -160,7 +171,12 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
                 if (lane == 0) {
                     ok = mbar_wait(bar_q_empty, (q_it & 1) ^ 1, s_abort, 202);
-                    if (ok) {
+                    if (ok && packed) {
+                        // rows = the G heads of this kv-head for the one token; rows G..127 keep whatever they held
+                        mbar_arrive_expect_tx(bar_q_full, 2 * G * 128);
+                        tma_load_3d(sQ, &tm_qh, bar_q_full, 0, h0, u.q_row0);
+                        tma_load_3d(sQ + kSlabBytes, &tm_qh, bar_q_full, 64, h0, u.q_row0);
+                    } else if (ok) {
                         mbar_arrive_expect_tx(bar_q_full, 2 * kTileBytes);
                         tma_load_4d(sQ, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0);
                         tma_load_4d(sQ + kTileBytes, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0 + 1);
@@ -256,7 +272,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
             constexpr uint32_t kIdescPV = idesc_bf16(128, 128, false, true);
             const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128, tO0 = tmem_base + 256, tO1 = tmem_base + 384;
-            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0;
+            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0, p_it1 = 0;   // p_it1: tile 1 sits packed items out
             auto wait1 = [&](uint32_t bar, uint32_t parity, int where) -> bool {
                 return mbar_wait(bar, parity, s_abort, where);
             };
@@ -284,6 +300,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!wait1(bar_item_full + 8 * slot, (item_it >> 1) & 1, 301)) break;
                 const WorkUnit u = ring[slot].u;
                 const int valid = ring[slot].valid;
+                const bool packed = ring[slot].packed != 0;
                 mbar_arrive(bar_item_empty + 8 * slot);
                 ++item_it;
                 if (!valid) break;
@@ -298,8 +315,10 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (lane == 0) {
                     issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                     tc_commit(bar_s_full);
-                    issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
-                    tc_commit(bar_s_full + 8);
+                    if (!packed) {
+                        issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
+                        tc_commit(bar_s_full + 8);
+                    }
                     tc_commit(bar_kv_empty + 8 * stK);
                     if (n == 1) tc_commit(bar_q_empty);
                 }
@@ -360,14 +379,25 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else if (lane == 0) {
                         tc_commit(bar_o_full);
                     }
+                    if (packed) {
+                        // no tile 1: the V stage and the next K stage are released here
+                        tc_commit(bar_kv_empty + 8 * stV);
+                        if (has_next) {
+                            tc_commit(bar_kv_empty + 8 * stK);
+                            if (jj + 2 == n) tc_commit(bar_q_empty);
+                            ++kv_it;
+                        }
+                        ++p_it;
+                        continue;
+                    }
                     // ---- tile 1 ----
                     if (kSplitChunks > 0) {
-                        ok = wait1(bar_p_part + 8, p_it & 1, 312);
+                        ok = wait1(bar_p_part + 8, p_it1 & 1, 312);
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 2 * kSplitChunks);
                     }
-                    ok = wait1(bar_p_full + 8, p_it & 1, 308);
+                    ok = wait1(bar_p_full + 8, p_it1 & 1, 308);
                     if (!ok) break;
                     tc_fence_after();
                     if (lane == 0) VPP_TR(0, jj, 5);
@@ -386,6 +416,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     if (lane == 0) VPP_TR(0, jj, 6);
                     if (has_next) ++kv_it;
                     ++p_it;
+                    ++p_it1;
                 }
                 if (!ok) break;
             }
@@ -415,14 +446,20 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             const uint32_t slot = item_it & 1;
             if (!mbar_wait(bar_item_full + 8 * slot, (item_it >> 1) & 1, s_abort, 401)) break;
             const WorkUnit u = ring[slot].u;
-            const int h = ring[slot].h0 + t;
+            const bool packed = ring[slot].packed != 0;
+            const int h = ring[slot].h0 + (packed ? row : t);   // packed: row r of tile 0 is q-head h0 + r
             const int valid = ring[slot].valid;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
             ++item_it;
             if (!valid) break;
+            if (packed && t == 1) continue;                     // tile 1 has no part in a packed item
+            // rows of this thread's warp that exist: a packed tile has G rows, a warp without any only keeps the
+            // barriers moving
+            const int tile_rows = packed ? G : u.rows;
+            const bool warp_idle = packed && (warp & 3) * 32 >= G;
 
-            const int my_pos = u.pos0 + row;
+            const int my_pos = packed ? u.pos0 : u.pos0 + row;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
             for (int j = u.kv_begin; j < u.kv_end; ++j) {
@@ -431,6 +468,15 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!ok) break;
                 ++s_it;
                 tc_fence_after();
+                if (warp_idle) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (kSplitChunks > 0) mbar_arrive(bar_p_part + 8 * t);
+                        mbar_arrive(bar_p);
+                    }
+                    continue;
+                }
                 if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 0);
                 uint32_t s[128];
                 const bool diag = tile0 + kTileN - 1 > u.pos0;  // keys beyond the row's position are masked
@@ -463,7 +509,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 const float m_new = fmaxf(mxa * sc, m_ref);
                 // lazy rescale: keep the old reference unless the maximum moved by more than 2^8
-                const bool grow = (m_new - m_ref > kRescaleThreshold) || (m_ref == -INFINITY && m_new != -INFINITY);
+                // (rows beyond the tile's last one hold leftovers: they never ask for a rescale)
+                const bool grow = row < tile_rows &&
+                                  ((m_new - m_ref > kRescaleThreshold) || (m_ref == -INFINITY && m_new != -INFINITY));
                 if (__any_sync(0xffffffffu, grow)) {
                     const float alpha = grow ? ex2(m_ref - m_new) : 1.f;  // m_ref = -inf gives 0
                     if (grow) m_ref = m_new;
@@ -522,8 +570,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             tc_fence_after();
             {
                 const float inv_l = 1.f / l_run;
-                const bool live = row < u.rows;
-                const long long grow_idx = static_cast<long long>(u.q_row0) + row;
+                const bool live = row < tile_rows;
+                const long long grow_idx = static_cast<long long>(u.q_row0) + (packed ? 0 : row);
                 uint32_t r[32];
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {

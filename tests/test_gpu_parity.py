@@ -103,6 +103,18 @@ def test_running_maximum_grows_every_tile(family, splits):
     print(s)
 
 
+@pytest.mark.parametrize("hq,hkv", [(64, 4), (16, 8), (8, 1)])
+@pytest.mark.parametrize("splits", [0, 1, 4])
+def test_decode_rows_mixed_with_prefill_chunks(hq, hkv, splits):
+    """Single-token requests (decode steps) batched with prefill chunks: the kernel packs the q-heads of a kv-head
+    into one tile for them.  Every element against the oracle."""
+    prefix = [700, 0, 1333, 128, 2047, 5, 300, 64, 1000]
+    chunk = [1, 1, 1, 1, 1, 1, 200, 129, 1]
+    prob = W.make_problem(2300 + hq, prefix, chunk, hq, hkv, 128, 128, block_size=16, std=0.7)
+    s, _ = full_check(prob, num_kv_splits=splits, label="decode mix Hq=%d Hkv=%d S=%d" % (hq, hkv, splits))
+    print(s)
+
+
 def test_mla_requires_aliased_values():
     prob = W.make_problem(2100, [10], [20], 2, 1, 576, 512, block_size=16, std=0.5, v_aliases_k=True).to("cuda")
     runner = api.ChunkAttn(prob)
