@@ -194,13 +194,68 @@ def bench_append(args):
     return 0
 
 
+def bench_decode(args):
+    """Decode rows (one query token per request) through the same attention entry point: HBM-bound, judged by the
+    bytes of K/V that have to be read once (context x Hkv x (Dqk + Dv) x 2 B) per second."""
+    import torch
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    cases = [("64 decode rows, context 32768, Hq=64 Hkv=8 d=128", [32768] * 64, [1] * 64, 64, 8),
+             ("64 decode rows, context 32768, Hq=64 Hkv=4 d=128", [32768] * 64, [1] * 64, 64, 4),
+             ("256 decode rows, context 8192, Hq=64 Hkv=8 d=128", [8192] * 256, [1] * 256, 64, 8),
+             ("16 decode rows (context 32768) + one 8192-token chunk at prefix 32768, Hq=64 Hkv=4", [32768] * 17,
+              [1] * 16 + [8192], 64, 4)]
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches = 0
+    for desc, prefix, chunk, hq, hkv in cases:
+        prob = W.make_problem(W.BASE_SEED + 91, prefix, chunk, hq, hkv, 128, 128, block_size=128, std=1.0, device=dev)
+        runner = api.ChunkAttn(prob)
+        kv_bytes = sum(p + c for p, c in zip(prefix, chunk)) * hkv * 256 * 2
+        n = max(args.steps, 5)
+        with torch.cuda.stream(stream):
+            for _ in range(max(args.warmup, 3)):
+                runner.run(stream.cuda_stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(n):
+                runner.run(stream.cuda_stream)
+            e1.record(stream)
+        e1.synchronize()
+        assert int(runner.status.item()) == 0
+        ms = e0.elapsed_time(e1) / n
+        launches += n * api.vpp_last_launch_count()
+        rows.append({"case": desc, "ms": round(ms, 4), "kv_GB/s": round(kv_bytes / ms / 1e6, 1),
+                     "frac_of_hbm_peak": round(kv_bytes / ms / 1e6 / peaks["hbm_gbs"], 4),
+                     "tflops": round(prob.flops() / ms / 1e9, 1), "kv_bytes": kv_bytes})
+        del prob, runner
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[0]
+    print(json.dumps({"metric": "decode rows through chunk attention: K/V GB/s vs HBM peak (1 B200)", "value": top["kv_GB/s"],
+                      "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic", "vs_baseline": None,
+                      "config": {"workload": "decode; " + top["case"], "l2": "K/V of every case exceeds the L2 (1 GB or more)"},
+                      "cases": rows,
+                      "roofline": {"bound": "hbm", "achieved": top["kv_GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": top["frac_of_hbm_peak"], "traffic": None,
+                                   "peak_source": "%s (copy bandwidth)" % peaks["_source"],
+                                   "kernel": "attn128_ws_kernel, packed single-token items; " + top["case"]},
+                      "gpu_launches": launches, "clocks": clocks}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -211,6 +266,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "append":
         return bench_append(args)
+    if args.workload == "decode":
+        return bench_decode(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,
