@@ -202,20 +202,27 @@ def bench_decode(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     peaks = load_peaks()
-    cases = [("64 decode rows, context 32768, Hq=64 Hkv=8 d=128", [32768] * 64, [1] * 64, 64, 8),
-             ("64 decode rows, context 32768, Hq=64 Hkv=4 d=128", [32768] * 64, [1] * 64, 64, 4),
-             ("256 decode rows, context 8192, Hq=64 Hkv=8 d=128", [8192] * 256, [1] * 256, 64, 8),
+    cases = [("64 decode rows, context 32768, Hq=64 Hkv=8 d=128", [32768] * 64, [1] * 64, 64, 8, 128),
+             ("64 decode rows, context 32768, Hq=64 Hkv=4 d=128", [32768] * 64, [1] * 64, 64, 4, 128),
+             ("256 decode rows, context 8192, Hq=64 Hkv=8 d=128", [8192] * 256, [1] * 256, 64, 8, 128),
              ("16 decode rows (context 32768) + one 8192-token chunk at prefix 32768, Hq=64 Hkv=4", [32768] * 17,
-              [1] * 16 + [8192], 64, 4)]
+              [1] * 16 + [8192], 64, 4, 128),
+             ("64 decode rows, context 32768, absorbed MLA Hq=128 (576/512), 64-token pages", [32768] * 64, [1] * 64, 128, 1, 576),
+             ("256 decode rows, context 8192, absorbed MLA Hq=128 (576/512), 64-token pages", [8192] * 256, [1] * 256, 128, 1, 576)]
     stream = torch.cuda.Stream()
     rows = []
     sampler = ClockSampler(0)
     sampler.start()
     launches = 0
-    for desc, prefix, chunk, hq, hkv in cases:
-        prob = W.make_problem(W.BASE_SEED + 91, prefix, chunk, hq, hkv, 128, 128, block_size=128, std=1.0, device=dev)
+    for desc, prefix, chunk, hq, hkv, dqk in cases:
+        if dqk == 128:
+            prob = W.make_problem(W.BASE_SEED + 91, prefix, chunk, hq, hkv, 128, 128, block_size=128, std=1.0, device=dev)
+            kv_bytes = sum(p + c for p, c in zip(prefix, chunk)) * hkv * 256 * 2
+        else:
+            prob = W.make_problem(W.BASE_SEED + 92, prefix, chunk, hq, 1, 576, 512, block_size=64, std=0.5,
+                                  scale=1.0 / 192 ** 0.5, v_aliases_k=True, device=dev)
+            kv_bytes = sum(p + c for p, c in zip(prefix, chunk)) * 576 * 2
         runner = api.ChunkAttn(prob)
-        kv_bytes = sum(p + c for p, c in zip(prefix, chunk)) * hkv * 256 * 2
         n = max(args.steps, 5)
         with torch.cuda.stream(stream):
             for _ in range(max(args.warmup, 3)):

@@ -331,7 +331,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_k2, a->k_cache, 5, d, sk, b5) || !make_tmap(&tm_v2, a->v_cache, 5, d, sv, b5))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
     }
-    CUtensorMap tm_q9, tm_k9;  // one 64-column slab of 64 rows per box
+    CUtensorMap tm_q9, tm_k9, tm_qh9;  // one 64-column slab of 64 rows per box
     const bool mla_pair = fam == Family::kMla576 && use_mla_pair_kernel(a);
     if (mla_pair) {
         const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), static_cast<uint64_t>(vpp::kMlaSlabs),
@@ -346,6 +346,13 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         const uint32_t b1[5] = {64, 64, 1, 1, 1};
         if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) || !make_tmap(&tm_k9, a->k_cache, 5, d, sk, b1))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");
+        // packed single-token items: 64 q-heads of one token as the rows of a CTA's Q tile
+        const uint64_t dh[4] = {64, static_cast<uint64_t>(a->num_q_heads), static_cast<uint64_t>(vpp::kMlaSlabs),
+                                static_cast<uint64_t>(a->total_q)};
+        const uint64_t sh[3] = {static_cast<uint64_t>(a->head_dim_qk) * 2, 128,
+                                static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2};
+        const uint32_t bh[4] = {64, static_cast<uint32_t>(a->num_q_heads < 64 ? a->num_q_heads : 64), 1, 1};
+        if (!make_tmap(&tm_qh9, a->q, 4, dh, sh, bh)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla q heads) failed");
     }
     CUtensorMap tm_k4, tm_k5;
     if (fam == Family::kMla576) {
@@ -410,7 +417,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     if (mla_pair) {
         auto kern = vpp::attn_mla2_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
-        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, ap);
+        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, tm_qh9, ap);
     } else if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);

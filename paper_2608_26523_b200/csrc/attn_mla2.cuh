@@ -148,7 +148,8 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMla2Threads, 1)
 attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_k1,
-                 const AttnParams p) {
+                 const __grid_constant__ CUtensorMap tm_qh, const AttnParams p) {
+    // tm_qh: (64 cols, Hq heads, 9 slabs, T rows) box (64, 64, 1, 1)      -- 64 q-heads of one token (packed items)
     // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 1, 1)         -- 64 query rows of one 64-column slab
     // tm_k1: (64 cols, keys, 9 slabs, head, block) box (64, 64, 1, 1, 1) -- 64 keys of one 64-column slab
     // Every tile is fetched slab by slab (8 KB copies).
@@ -208,6 +209,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         *s_abort = 0;
         prefetch_tmap(&tm_q1);
         prefetch_tmap(&tm_k1);
+        prefetch_tmap(&tm_qh);
     }
     __syncthreads();
     cluster_sync_all();  // barrier initialisation is visible to the other CTA before anything arrives remotely
@@ -221,20 +223,33 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
     const uint32_t tmem_base = *s_tmem;
 
     const int num_units = p.header_ro->num_units;
-    const int total_items = num_units * p.num_q_heads;
     const int num_pairs = gridDim.x >> 1;
     const int pair = blockIdx.x >> 1;
+    // Items: (unit, q-head) for the units of several rows, then one item per single-token unit (the end of the list):
+    // those run "packed" -- the q-heads are the rows of the tile (64 per CTA; they all share the one latent kv-head), so
+    // the cache is streamed once per token instead of once per head.
+    const int num_packed = p.num_q_heads <= 2 * kMla2Rows ? p.header_ro->num_single : 0;
+    const int num_normal = num_units - num_packed;
+    const int normal_items = num_normal * p.num_q_heads;
+    const int total_items = normal_items + num_packed;
 
     // KV tiles (128 keys) of a unit: [kv_begin, min(kv_end, ceil((pos0 + rows) / 128)))
     auto tile_hi = [](const WorkUnit& u) {
         const int need = (u.pos0 + u.rows + kTileN - 1) / kTileN;
         return u.kv_end < need ? u.kv_end : need;
     };
-    auto get_item = [&](int item, WorkUnit& u, int& h) {
-        int ui;
-        decode_item(item, num_units, p.num_q_heads, p.num_q_heads, ui, h);
-        u = p.units[ui];
+    auto get_item = [&](int item, WorkUnit& u, int& h) -> bool {
+        if (item < normal_items) {
+            int ui;
+            decode_item(item, num_normal, p.num_q_heads, p.num_q_heads, ui, h);
+            u = p.units[ui];
+        } else {
+            u = p.units[num_normal + (item - normal_items)];
+            h = 0;
+        }
+        return true;
     };
+    auto is_packed = [&](const WorkUnit& u) { return num_packed > 0 && u.rows == 1; };
     // page and slot of the 64-key group that starts at position pos
     auto page_of = [&](const WorkUnit& u, int pos, int& blk, int& slot_in) {
         if (p.block_table == nullptr) {
@@ -278,15 +293,21 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             for (int item = pair; item < total_items && ok; item += num_pairs) {
                 WorkUnit u;
                 int h;
-                get_item(item, u, h);
+                if (!get_item(item, u, h)) continue;
                 ++item_it;
                 // Q may be replaced once the scores of the previous item's last tile are done
                 if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 801);
                 if (!ok) break;
-                if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMla2QBytes);
+                // (a packed tile has min(64, Hq) rows per CTA; rows of a copy that lie outside the tensor still count)
+                const int q_rows = is_packed(u) ? (p.num_q_heads < kMla2Rows ? p.num_q_heads : kMla2Rows) : kMla2Rows;
+                if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMlaSlabs * q_rows * 128);
 #pragma unroll 1
-                for (int s = 0; s < kMlaSlabs; ++s)
-                    tma2_load_4d(sQ + s * 8192, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, s, h);
+                for (int s = 0; s < kMlaSlabs; ++s) {
+                    if (is_packed(u))   // heads 64 rank .. 64 rank + 63 of the token (heads that do not exist read as zero)
+                        tma2_load_4d(sQ + s * 8192, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, s, u.q_row0);
+                    else
+                        tma2_load_4d(sQ + s * 8192, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, s, h);
+                }
                 ++q_it;
                 const int t_hi = tile_hi(u);
                 int blk_next = 0, slot_next = 0;
@@ -323,7 +344,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
-            get_item(item, u, h);
+            if (!get_item(item, u, h)) continue;
             const int t_hi = tile_hi(u);
             int nb0 = 0, ns0 = 0, nb1 = 0, ns1 = 0;
             if (lane == 0) {
@@ -423,7 +444,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
-            get_item(item, u, h);
+            if (!get_item(item, u, h)) continue;
             const int n = tile_hi(u) - u.kv_begin;
             ++item_it;
             ok = mbar_wait(bar_q_full, q_it & 1, s_abort, 821);
@@ -507,11 +528,13 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
-            get_item(item, u, h);
+            if (!get_item(item, u, h)) continue;
             const int t_hi = tile_hi(u);
             ++item_it;
             const int my_row = static_cast<int>(rank) * kMla2Rows + row;  // row of the 128-row tile
-            const int my_pos = u.pos0 + my_row;
+            const bool packed = is_packed(u);
+            const int my_pos = packed ? u.pos0 : u.pos0 + my_row;
+            if (packed) h = my_row;                                       // row r of a packed tile is q-head r
             float m_ref = -INFINITY, l_run = 0.f;
             for (int j = u.kv_begin; j < t_hi; ++j) {
                 const int tile0 = j * kTileN;
@@ -613,8 +636,8 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             if (!ok) break;
             tc_fence_after();
             const float inv_l = 1.f / l_tot;
-            const bool live = my_row < u.rows;
-            const long long grow_idx = static_cast<long long>(u.q_row0) + my_row;
+            const bool live = packed ? my_row < p.num_q_heads : my_row < u.rows;
+            const long long grow_idx = static_cast<long long>(u.q_row0) + (packed ? 0 : my_row);
             uint32_t r[32];
 #pragma unroll 1
             for (int c = 0; c < 8; ++c) {

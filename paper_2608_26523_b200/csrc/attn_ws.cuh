@@ -130,7 +130,12 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     const int num_units = p.header_ro->num_units;
     const int G = p.num_q_heads / p.num_kv_heads;
-    const int total_items = num_units * (p.num_q_heads / 2);
+    // Items: (unit, pair of q-heads) for the units of several rows, then (unit, kv-head) for the single-token units at the
+    // end of the list, which run packed when a kv-head's group fits a tile.
+    const int num_packed = G <= kTileM ? p.header_ro->num_single : 0;
+    const int num_normal = num_units - num_packed;
+    const int normal_items = num_normal * (p.num_q_heads / 2);
+    const int total_items = normal_items + num_packed * p.num_kv_heads;
 
     if (warp < 4) {
         if (warp == 0) {
@@ -144,14 +149,16 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 WorkUnit u{};
                 int h0 = 0;
                 bool packed = false;
-                if (have) {
+                if (have && item < normal_items) {
                     int ui, hp;
-                    decode_item(item, num_units, p.num_q_heads / 2, G / 2, ui, hp);
+                    decode_item(item, num_normal, p.num_q_heads / 2, G / 2, ui, hp);
                     u = p.units[ui];
                     h0 = 2 * hp;
-                    packed = u.rows == 1 && G <= kTileM;
-                    // a packed unit is served by the first head slot of each kv-head; its other slots have nothing to do
-                    if (packed && h0 % G != 0) continue;
+                } else if (have) {
+                    const int k = item - normal_items;
+                    u = p.units[num_normal + k / p.num_kv_heads];
+                    h0 = (k % p.num_kv_heads) * G;
+                    packed = true;
                 }
                 const uint32_t slot = item_it & 1;
                 bool ok = true;

@@ -26,7 +26,7 @@ struct WorkHeader {
     int32_t num_units;  // units in the sorted list
     int32_t counter;    // persistent-kernel work counter
     int32_t error;      // VPP_DEV_* (0 = ok); when nonzero num_units is 0
-    int32_t pad;
+    int32_t num_single; // the last num_single units of the list are single-token units (rows == 1)
 };
 
 struct WorkspaceLayout {

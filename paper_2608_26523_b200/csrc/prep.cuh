@@ -85,7 +85,7 @@ __device__ __forceinline__ int cost_bin(int cost, int max_cost) {
 
 __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams p) {
     __shared__ int warp_sums[33];
-    __shared__ int bins[kCostBins];
+    __shared__ int bins[2 * kCostBins];   // [0, kCostBins): units of several rows; [kCostBins, ..): single-token units
     __shared__ int s_error;
     __shared__ int s_carry_q, s_carry_t;
     const int tid = threadIdx.x;
@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
         s_carry_q = 0;
         s_carry_t = 0;
     }
-    for (int b = tid; b < kCostBins; b += kPrepThreads) bins[b] = 0;
+    for (int b = tid; b < 2 * kCostBins; b += kPrepThreads) bins[b] = 0;
     __syncthreads();
 
     // ---- phase 1: validate lengths, scan chunk lengths and query-tile counts over requests ----
@@ -152,6 +152,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
     if (s_error != 0) {
         if (tid == 0) {
             p.header->num_units = 0;
+            p.header->num_single = 0;
             p.header->counter = 0;
             p.header->error = s_error;
             if (p.status) *p.status = s_error;
@@ -179,7 +180,9 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
             for (int s = 0; s < nsplit; ++s) {
                 int kb, ke;
                 split_range(pos0, n_tiles, nsplit, s, kb, ke);
-                const int bin = cost_bin(ke - kb, p.max_cost);
+                // single-token units go to the end of the list (each part ordered by decreasing cost): the attention
+                // kernels may run them with the q-heads of a kv-head packed into one tile
+                const int bin = cost_bin(ke - kb, p.max_cost) + (rows == 1 ? kCostBins : 0);
                 if (pass == 0) {
                     atomicAdd(&bins[bin], 1);
                 } else {
@@ -205,14 +208,20 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
         __syncthreads();
         if (pass == 0) {
             // exclusive scan of the bins (bin 0 = most expensive first)
-            static_assert(kCostBins == 2 * kPrepThreads, "two bins per thread");
-            const int a = bins[2 * tid], b = bins[2 * tid + 1];
+            static_assert(2 * kCostBins == 4 * kPrepThreads, "four bins per thread");
+            const int b0 = bins[4 * tid], b1 = bins[4 * tid + 1], b2 = bins[4 * tid + 2], b3 = bins[4 * tid + 3];
             int total;
-            const int ex = block_exclusive_scan(a + b, warp_sums, total);
-            bins[2 * tid] = ex;
-            bins[2 * tid + 1] = ex + a;
+            const int ex = block_exclusive_scan(b0 + b1 + b2 + b3, warp_sums, total);
+            bins[4 * tid] = ex;
+            bins[4 * tid + 1] = ex + b0;
+            bins[4 * tid + 2] = ex + b0 + b1;
+            bins[4 * tid + 3] = ex + b0 + b1 + b2;
+            __syncthreads();
             if (tid == 0) {
-                p.header->num_units = total < p.max_units ? total : p.max_units;
+                const int n = total < p.max_units ? total : p.max_units;
+                const int first_single = bins[kCostBins] < n ? bins[kCostBins] : n;
+                p.header->num_units = n;
+                p.header->num_single = n - first_single;
                 p.header->counter = 0;
                 p.header->error = 0;
                 if (p.status) *p.status = 0;

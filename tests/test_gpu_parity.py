@@ -115,6 +115,18 @@ def test_decode_rows_mixed_with_prefill_chunks(hq, hkv, splits):
     print(s)
 
 
+@pytest.mark.parametrize("hq", [128, 16, 72])
+@pytest.mark.parametrize("splits", [0, 1, 4])
+def test_mla_decode_rows_mixed_with_prefill_chunks(hq, splits):
+    """Absorbed MLA: single-token requests next to prefill chunks (the q-heads become the rows of the tile)."""
+    prefix = [700, 0, 1333, 128, 2047, 5, 300, 64]
+    chunk = [1, 1, 1, 1, 1, 1, 130, 1]
+    prob = W.make_problem(2400 + hq, prefix, chunk, hq, 1, 576, 512, block_size=64, std=0.5, scale=1.0 / 192 ** 0.5,
+                          v_aliases_k=True)
+    s, _ = full_check(prob, num_kv_splits=splits, label="mla decode mix Hq=%d S=%d" % (hq, splits))
+    print(s)
+
+
 def test_mla_requires_aliased_values():
     prob = W.make_problem(2100, [10], [20], 2, 1, 576, 512, block_size=16, std=0.5, v_aliases_k=True).to("cuda")
     runner = api.ChunkAttn(prob)
