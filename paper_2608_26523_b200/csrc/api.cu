@@ -425,7 +425,21 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     } else if (use_ws_kernel(a)) {
         auto kern = vpp::attn128_ws_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kWsThreads, vpp::kWsSmemBytes, stream>>>(tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, tm_qh, ap, box_rows);
+        if (ce == cudaSuccess) {
+            // programmatic dependent launch: set-up overlaps the work-decomposition kernel (the kernel waits for it
+            // before it reads the work list)
+            cudaLaunchAttribute attr{};
+            attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr.val.programmaticStreamSerializationAllowed = 1;
+            cudaLaunchConfig_t cfg{};
+            cfg.gridDim = dim3(sms);
+            cfg.blockDim = dim3(vpp::kWsThreads);
+            cfg.dynamicSmemBytes = vpp::kWsSmemBytes;
+            cfg.stream = stream;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            ce = cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, tm_qh, ap, box_rows);
+        }
     } else {
         auto kern = vpp::attn128_simple_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);
@@ -439,9 +453,21 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         const long long pairs = static_cast<long long>(a->total_q) * a->num_q_heads;
         long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
         if (blocks > 8ll * sms) blocks = 8ll * sms;
-        vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
-            ap.o_parts, ap.lse_parts, L.splits, a->total_q, a->num_q_heads, a->head_dim_v, row_splits,
-            static_cast<__nv_bfloat16*>(a->out), a->lse);
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+        cfg.blockDim = dim3(vpp::kMergeThreads);
+        cfg.stream = stream;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        ce = cudaLaunchKernelEx(&cfg, vpp::lse_merge_kernel, static_cast<const float*>(ap.o_parts),
+                                static_cast<const float*>(ap.lse_parts), static_cast<int>(L.splits),
+                                static_cast<long long>(a->total_q), static_cast<int>(a->num_q_heads),
+                                static_cast<int>(a->head_dim_v), static_cast<const int32_t*>(row_splits),
+                                static_cast<__nv_bfloat16*>(a->out), a->lse);
+        if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "merge launch: %s", cudaGetErrorString(ce));
         ++g_launches;
     }
     ce = cudaGetLastError();

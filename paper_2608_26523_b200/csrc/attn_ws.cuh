@@ -128,6 +128,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
 
+    pdl_wait();                  // the work list comes from the work-decomposition kernel launched just before
+    pdl_launch_dependents();     // (the merge kernel, if any, waits for this grid to finish in the same way)
     const int num_units = p.header_ro->num_units;
     const int G = p.num_q_heads / p.num_kv_heads;
     // Items: (unit, pair of q-heads) for the units of several rows, then (unit, kv-head) for the single-token units at the

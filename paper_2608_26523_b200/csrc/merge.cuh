@@ -23,6 +23,7 @@ __global__ void __launch_bounds__(kMergeThreads)
 lse_merge_kernel(const float* __restrict__ o_parts, const float* __restrict__ lse_parts, int num_splits,
                  long long total_q, int num_q_heads, int head_dim_v, const int32_t* __restrict__ row_splits,
                  __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // partials come from the attention kernel launched just before
     const long long n_pairs = total_q * num_q_heads;
     const int lane = threadIdx.x & 31;
     const long long warps_total = static_cast<long long>(gridDim.x) * (kMergeThreads / 32);

@@ -7,6 +7,7 @@
 // which is the per-chunk imbalance the paper's Eq. 2 models.
 #pragma once
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace vpp {
 
@@ -89,6 +90,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
     __shared__ int s_error;
     __shared__ int s_carry_q, s_carry_t;
     const int tid = threadIdx.x;
+    pdl_launch_dependents();   // the attention kernel may set itself up (barriers, tensor memory) while this runs
     if (tid == 0) {
         s_error = 0;
         s_carry_q = 0;

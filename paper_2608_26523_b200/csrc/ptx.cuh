@@ -264,6 +264,12 @@ __device__ __forceinline__ float ex2_poly(float x) {
     p = fmaf(p, f, 1.0000026226043701f);
     return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xf) << 23));
 }
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization attribute may start
+// while its predecessor in the stream still runs; pdl_wait() returns once that predecessor has completed and its
+// writes are visible.  pdl_launch_dependents() lets the successor's blocks be scheduled from now on.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // three-input maximum (one instruction on sm_100)
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float r;
