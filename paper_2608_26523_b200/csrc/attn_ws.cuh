@@ -14,13 +14,17 @@
 //   warps 8-11  the same for tile 1.
 // While one group works on its S tile the tensor core runs the other tile's MMAs.
 // A work unit of a single query token (a decode step batched with prefill chunks, or the one-row tail of a chunk) is
-// run "packed": the G q-heads that share a kv-head become the rows of tile 0, so its K/V is streamed once per
-// kv-head instead of once per pair of q-heads; tile 1 and its softmax group sit the item out.
+// run "packed": the G q-heads that share a kv-head become the rows of the Q tile, so its K/V is streamed once per
+// kv-head instead of once per pair of q-heads.  Both tiles then use that one Q tile and split the KV tiles between
+// them (even ones to tile 0, odd ones to tile 1) as two independent online softmaxes whose results softmax group 0
+// merges at the end -- one softmax chain per KV tile would leave the memory system idle most of the time.
 // Tensor memory: S_0 | S_1 | O_0 | O_1, 128 fp32 columns each (all 512 columns).
 //
 // The math per row is the paper's Eq. 1 with the causal rule, evaluated KV tile by KV tile with a
 // running maximum; O is rescaled lazily (only when the maximum has grown by more than 2^8).
 #pragma once
+#include <type_traits>
+
 #include "attn_simple.cuh"  // decode_item, kSlabBytes
 #include "common.cuh"
 #include "ptx.cuh"
@@ -33,7 +37,7 @@ constexpr int kWsThreads = 384;
 #endif
 constexpr int kWsStages = VPP_WS_STAGES;      // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
-constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 1024 /*barriers, ring*/;
+constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 2048 /*barriers, ring, merge exchange*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
 #ifndef VPP_SPLIT_CHUNKS
 #define VPP_SPLIT_CHUNKS 1
@@ -54,6 +58,64 @@ struct WsItem {
     int32_t pad;
 };
 
+
+// Merge of the two tiles' partial results of a packed item (rare path, kept out of line to spare the main loop's
+// registers):  out = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1),  a_t = 2^(m_t - m).  O_1 sits 128 columns after O_0.
+// (every argument by value: a reference to the kernel's parameter block or to the work unit would force them into
+// local memory for the whole kernel)
+__device__ __noinline__ void ws_packed_merge(void* out, float* lse_out, float* o_parts, float* lse_parts, int total_q,
+                                             int num_q_heads, int split, int q_row0, bool second, const float* xm,
+                                             uint32_t tO, int row, int tile_rows, int h, float m_ref, float l_run) {
+    const float m1 = xm[row], l1 = xm[128 + row];
+    const float m = fmaxf(m_ref, m1);
+    const float a0 = m_ref == -INFINITY ? 0.f : ex2(m_ref - m), a1 = m1 == -INFINITY ? 0.f : ex2(m1 - m);
+    const float l_tot = a0 * l_run + a1 * l1;
+    const float s0 = a0 / l_tot, s1 = a1 / l_tot;
+    const bool live = row < tile_rows;
+    const long long grow_idx = q_row0;
+    uint32_t r[16], r1[16];
+#pragma unroll 1
+    for (int c = 0; c < 8; ++c) {     // 16 output columns at a time (registers)
+        tmem_ld16(tO + c * 16, r);
+        if (second) tmem_ld16(tO + 128 + c * 16, r1);
+        tc_wait_ld();
+        if (!live) continue;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            float v = __uint_as_float(r[i]) * s0;
+            if (second) v = fmaf(__uint_as_float(r1[i]), s1, v);
+            r[i] = __float_as_uint(v);
+        }
+        if (split < 0) {
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(out) +
+                                                  ((grow_idx * num_q_heads + h) * 128 + c * 16) * 2);
+#pragma unroll
+            for (int q4 = 0; q4 < 2; ++q4) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    w[e] = pack_bf16x2(__uint_as_float(r[q4 * 8 + 2 * e]), __uint_as_float(r[q4 * 8 + 2 * e + 1]));
+                dst[q4] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        } else {
+            float4* dst = reinterpret_cast<float4*>(
+                o_parts +
+                ((static_cast<long long>(split) * total_q + grow_idx) * num_q_heads + h) * 128 + c * 16);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)
+                dst[q4] = make_float4(__uint_as_float(r[q4 * 4]), __uint_as_float(r[q4 * 4 + 1]),
+                                      __uint_as_float(r[q4 * 4 + 2]), __uint_as_float(r[q4 * 4 + 3]));
+        }
+    }
+    if (live) {
+        const float lse = (m + log2f(l_tot)) * 0.6931471805599453f;
+        if (split < 0) {
+            if (lse_out) lse_out[grow_idx * num_q_heads + h] = lse;
+        } else {
+            lse_parts[(static_cast<long long>(split) * total_q + grow_idx) * num_q_heads + h] = lse;
+        }
+    }
+}
 
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -83,10 +145,13 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_p_part = sBar + 104;      // [2] first kSplitCols key columns of P are in place (optional early hand-off)
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
     const uint32_t bar_kv_empty = sBar + 128 + 8 * kWsStages;
+    const uint32_t bar_x1 = sBar + 128 + 16 * kWsStages;       // packed item: group 1 has published its (m, l) per row
+    const uint32_t bar_x0 = sBar + 128 + 16 * kWsStages + 8;   // packed item: group 0 has merged, tile 1 may be reused
     uint8_t* gen_bar = gen_base + (2 + kWsStages) * kTileBytes;
     volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 512);
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 516);
     WsItem* ring = reinterpret_cast<WsItem*>(gen_bar + 576);  // 2 x 48 bytes
+    float* xm = reinterpret_cast<float*>(gen_bar + 1024);     // [2][128]: running maximum and row sum of tile 1 (packed items)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -104,6 +169,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(bar_q_full, 1);
         mbar_init(bar_q_empty, 1);
         mbar_init(bar_vfix, 1);
+        mbar_init(bar_x1, 4);
+        mbar_init(bar_x0, 4);
         for (int i = 0; i < kWsStages; ++i) {
             mbar_init(bar_kv_full + 8 * i, 1);
             mbar_init(bar_kv_empty + 8 * i, 1);
@@ -281,7 +348,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
             constexpr uint32_t kIdescPV = idesc_bf16(128, 128, false, true);
             const uint32_t tS0 = tmem_base, tS1 = tmem_base + 128, tO0 = tmem_base + 256, tO1 = tmem_base + 384;
-            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0, p_it1 = 0;   // p_it1: tile 1 sits packed items out
+            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_it = 0, p_it = 0, p_it1 = 0;   // P hand-offs seen per tile
             auto wait1 = [&](uint32_t bar, uint32_t parity, int where) -> bool {
                 return mbar_wait(bar, parity, s_abort, where);
             };
@@ -316,6 +383,57 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 const int n = u.kv_end - u.kv_begin;
                 if (!wait1(bar_q_full, q_it & 1, 302)) break;
                 ++q_it;
+                if (packed) {
+                    // Packed single-token item: both tiles hold the same Q (the heads of one kv-head) and share the KV
+                    // range -- tile t takes the KV tiles kv_begin + t, + t + 2, ... as an independent online softmax
+                    // (its own S_t, O_t); the two partial results are merged by softmax group 0 at the end.
+                    // Ring index of K(jj) is base + 2 jj, of V(jj) base + 2 jj + 1.
+                    const uint32_t base = kv_it;
+                    bool ok = true;
+                    auto do_qk = [&](int jj) {
+                        const uint32_t idx = base + 2 * jj, st = idx % kWsStages;
+                        if (!wait1(bar_kv_full + 8 * st, (idx / kWsStages) & 1, 321)) return false;
+                        tc_fence_after();
+                        issue_qk((jj & 1) ? tS1 : tS0, q_lo0, sKV + st * kTileBytes);
+                        tc_commit(bar_s_full + 8 * (jj & 1));
+                        tc_commit(bar_kv_empty + 8 * st);
+                        if (jj + 1 == n) tc_commit(bar_q_empty);
+                        return true;
+                    };
+                    ok = do_qk(0);
+                    if (ok && n > 1) ok = do_qk(1);
+                    for (int jj = 0; jj < n && ok; ++jj) {
+                        const int t = jj & 1;
+                        const int tile0 = (u.kv_begin + jj) * kTileN;
+                        const uint32_t idx = base + 2 * jj + 1, st = idx % kWsStages;
+                        const uint32_t pit = t ? p_it1 : p_it;   // (no reference: the counters must stay in registers)
+                        ok = wait1(bar_kv_full + 8 * st, (idx / kWsStages) & 1, 322);
+                        if (!ok) break;
+                        if (tile0 + kTileN > u.kv_len) {
+                            ok = wait1(bar_vfix, vfix_it & 1, 323);
+                            if (!ok) break;
+                            ++vfix_it;
+                        }
+                        const uint32_t tO = t ? tO1 : tO0, tS = t ? tS1 : tS0;
+                        if (kSplitChunks > 0) {
+                            ok = wait1(bar_p_part + 8 * t, pit & 1, 324);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(tO, tS, sKV + st * kTileBytes, jj < 2, 0, 2 * kSplitChunks);
+                        }
+                        ok = wait1(bar_p_full + 8 * t, pit & 1, 325);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(tO, tS, sKV + st * kTileBytes, jj < 2, kSplitChunks > 0 ? 2 * kSplitChunks : 0, 8);
+                        tc_commit(bar_kv_empty + 8 * st);
+                        if (t) ++p_it1; else ++p_it;
+                        if (jj + 2 < n) ok = do_qk(jj + 2);
+                        else tc_commit(bar_o_full + 8 * t);     // this tile's last KV tile
+                    }
+                    if (!ok) break;
+                    kv_it = base + 2 * n;
+                    continue;
+                }
                 // S_t(0) = Q_t K(0)^T
                 uint32_t stK = kv_it % kWsStages;
                 if (!wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 303)) break;
@@ -324,10 +442,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (lane == 0) {
                     issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                     tc_commit(bar_s_full);
-                    if (!packed) {
-                        issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
-                        tc_commit(bar_s_full + 8);
-                    }
+                    issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
+                    tc_commit(bar_s_full + 8);
                     tc_commit(bar_kv_empty + 8 * stK);
                     if (n == 1) tc_commit(bar_q_empty);
                 }
@@ -388,17 +504,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else if (lane == 0) {
                         tc_commit(bar_o_full);
                     }
-                    if (packed) {
-                        // no tile 1: the V stage and the next K stage are released here
-                        tc_commit(bar_kv_empty + 8 * stV);
-                        if (has_next) {
-                            tc_commit(bar_kv_empty + 8 * stK);
-                            if (jj + 2 == n) tc_commit(bar_q_empty);
-                            ++kv_it;
-                        }
-                        ++p_it;
-                        continue;
-                    }
                     // ---- tile 1 ----
                     if (kSplitChunks > 0) {
                         ok = wait1(bar_p_part + 8, p_it1 & 1, 312);
@@ -449,7 +554,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const uint32_t tS = tmem_base + t * 128 + lane_off;
         const uint32_t tO = tmem_base + 256 + t * 128 + lane_off;
         const uint32_t bar_s = bar_s_full + 8 * t, bar_p = bar_p_full + 8 * t, bar_o = bar_o_full + 8 * t;
-        uint32_t item_it = 0, s_it = 0, o_it = 0;
+        uint32_t item_it = 0, s_it = 0, o_it = 0, x_it = 0;
         const float sc = p.scale_log2e;
         while (true) {
             const uint32_t slot = item_it & 1;
@@ -462,16 +567,20 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
             ++item_it;
             if (!valid) break;
-            if (packed && t == 1) continue;                     // tile 1 has no part in a packed item
+            // One item's softmax work.  The packed variant (single-token items) is compiled separately so that the
+            // prefill path keeps the registers and the instruction count it had without it.
+            auto run_item = [&](auto packed_tag) -> bool {
+            constexpr bool kPacked = decltype(packed_tag)::value;
             // rows of this thread's warp that exist: a packed tile has G rows, a warp without any only keeps the
             // barriers moving
-            const int tile_rows = packed ? G : u.rows;
-            const bool warp_idle = packed && (warp & 3) * 32 >= G;
+            const int tile_rows = kPacked ? G : u.rows;
+            const bool warp_idle = kPacked && (warp & 3) * 32 >= G;
 
-            const int my_pos = packed ? u.pos0 : u.pos0 + row;
+            const int my_pos = kPacked ? u.pos0 : u.pos0 + row;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
-            for (int j = u.kv_begin; j < u.kv_end; ++j) {
+            // a packed item: this group's tile takes every second KV tile
+            for (int j = u.kv_begin + (kPacked ? t : 0); j < u.kv_end; j += kPacked ? 2 : 1) {
                 const int tile0 = j * kTileN;
                 ok = mbar_wait(bar_s, s_it & 1, s_abort, 402);
                 if (!ok) break;
@@ -525,7 +634,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const float alpha = grow ? ex2(m_ref - m_new) : 1.f;  // m_ref = -inf gives 0
                     if (grow) m_ref = m_new;
                     l_run *= alpha;
-                    if (j > u.kv_begin) {
+                    if (j > u.kv_begin + (kPacked ? t : 0)) {   // O of this tile already holds something
                         uint32_t o[32];
 #pragma unroll 1
                         for (int c = 0; c < 4; ++c) {
@@ -570,17 +679,45 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p);
             }
-            if (!ok) break;
+            if (!ok) return false;
 
             // ---- epilogue ----
-            ok = mbar_wait(bar_o, o_it & 1, s_abort, 403);
-            if (!ok) break;
-            ++o_it;
+            const bool have_tiles = !kPacked || u.kv_begin + t < u.kv_end;   // (tile 1 of a one-tile packed item has none)
+            if (have_tiles) {
+                ok = mbar_wait(bar_o, o_it & 1, s_abort, 403);
+                if (!ok) return false;
+                ++o_it;
+            }
             tc_fence_after();
+            if (kPacked && t == 1) {
+                // hand (m, l) of every row to group 0, which also reads O_1; wait until it is done with them
+                xm[row] = m_ref;
+                xm[128 + row] = l_run;
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_x1);
+                ok = mbar_wait(bar_x0, x_it & 1, s_abort, 404);
+                if (!ok) return false;
+                ++x_it;
+                return true;
+            }
+            if (kPacked) {
+                // merge the two tiles' partial results:  out = (a0 O_0 + a1 O_1) / (a0 l_0 + a1 l_1),  a_t = 2^(m_t - m)
+                ok = mbar_wait(bar_x1, x_it & 1, s_abort, 405);
+                if (!ok) return false;
+                ++x_it;
+                tc_fence_after();
+                ws_packed_merge(p.out, p.lse, p.o_parts, p.lse_parts, p.total_q, p.num_q_heads, u.split, u.q_row0,
+                                u.kv_begin + 1 < u.kv_end /* O_1 was written at all */, xm, tO, row, tile_rows, h, m_ref, l_run);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_x0);
+                return true;
+            }
             {
                 const float inv_l = 1.f / l_run;
                 const bool live = row < tile_rows;
-                const long long grow_idx = static_cast<long long>(u.q_row0) + (packed ? 0 : row);
+                const long long grow_idx = static_cast<long long>(u.q_row0) + row;
                 uint32_t r[32];
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
@@ -620,6 +757,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             }
             tc_fence_before();
+            return true;
+            };
+            if (!(packed ? run_item(std::true_type{}) : run_item(std::false_type{}))) break;
         }
     }
 
