@@ -28,6 +28,8 @@
 // on the item sequence without exchanging anything.
 // The math per row is the paper's Eq. 1 with the causal rule, KV tile by KV tile with a running maximum.
 #pragma once
+#include <type_traits>
+
 #include "attn_mla.cuh"  // kMla* constants
 #include "common.cuh"
 #include "ptx.cuh"
@@ -417,8 +419,11 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         bool ok = true;
         // scores of K group g (kKG slabs) into tS; the group goes back to the producer when its MMAs are done and
         // the last group's commit also tells the softmax warps that the scores are complete
-        auto qk_group = [&](uint32_t tS, int g, uint32_t bar_last) {
-#pragma unroll 1
+        // The issuing thread has nothing to hide instruction latency behind, so the groups are unrolled completely with
+        // compile-time offsets: every descriptor is (a loop-invariant base) + (a constant).
+        auto qk_group_c = [&](auto gc, uint32_t tS, uint32_t bar_last) {
+            constexpr int g = decltype(gc)::value;
+#pragma unroll
             for (int s = g * kKG; s < (g + 1) * kKG; ++s) {
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
@@ -428,9 +433,17 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             }
             tc_commit2(g < kKGroups - 1 ? bar_k_empty + 8 * g : bar_last, 3);
         };
+        auto qk_group = [&](uint32_t tS, int g, uint32_t bar_last) {
+            static_assert(kKGroups == 3, "one case per K group");
+            if (g == 0) qk_group_c(std::integral_constant<int, 0>{}, tS, bar_last);
+            else if (g == 1) qk_group_c(std::integral_constant<int, 1>{}, tS, bar_last);
+            else qk_group_c(std::integral_constant<int, 2>{}, tS, bar_last);
+        };
         // O += P V for V group g: chunk c = (key half c >> 1, output half c & 1)
-        auto pv_group = [&](int g, bool first_tile) {
-#pragma unroll 1
+        auto pv_group_c = [&](auto gc, auto firstc) {
+            constexpr int g = decltype(gc)::value;
+            constexpr bool first_tile = decltype(firstc)::value;
+#pragma unroll
             for (int c = g * kVG; c < (g + 1) * kVG; ++c) {
                 const uint32_t tO = (c & 1) ? tO1 : tO0;
 #pragma unroll
@@ -440,6 +453,16 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 }
             }
             tc_commit2(g < kVGroups - 1 ? bar_v_empty + 8 * g : bar_pv_done, 3);
+        };
+        auto pv_group = [&](int g, bool first_tile) {
+            static_assert(kVGroups == 2, "one case per V group");
+            if (g == 0) {
+                if (first_tile) pv_group_c(std::integral_constant<int, 0>{}, std::true_type{});
+                else pv_group_c(std::integral_constant<int, 0>{}, std::false_type{});
+            } else {
+                if (first_tile) pv_group_c(std::integral_constant<int, 1>{}, std::true_type{});
+                else pv_group_c(std::integral_constant<int, 1>{}, std::false_type{});
+            }
         };
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
