@@ -10,9 +10,10 @@
 // 256 value columns of each P V instruction (128 each) -- so each K/V byte is fetched from L2 once per 128
 // query rows without any multicast copy.
 //
-// Per CTA, 7 warps:
+// Per CTA, 8 warps:
 //   warp 0      one thread: Q and K producer (TMA); the warp also allocates tensor memory
-//   warp 1      rank 0: the one thread that issues every MMA of the pair and the multicast commits; rank 1: idle
+//   warp 1      rank 0: the thread that issues the score MMAs of the pair and their multicast commits; rank 1: idle
+//   warp 7      rank 0: the thread that issues the P V MMAs of the pair; rank 1: idle
 //   warps 2-5   softmax: lane l of tensor memory holds 64 score columns of row l & 63; the two threads of a row
 //               exchange their row maximum through shared memory; P goes to shared memory (K-major, 128B swizzle)
 //   warp 6      V producer (TMA) and zero-fill of value rows past the end of the sequence
@@ -36,7 +37,7 @@
 
 namespace vpp {
 
-constexpr int kMla2Threads = 224;
+constexpr int kMla2Threads = 256;
 constexpr int kMla2Rows = 64;                                 // query rows per CTA
 constexpr int kMla2QBytes = kMlaSlabs * kMla2Rows * 128;      // 72 KB: 9 slabs x 64 rows
 constexpr int kMla2KBytes = kMlaSlabs * 64 * 128;             // 72 KB: 9 slabs x 64 keys (this CTA's half of a tile)
@@ -408,19 +409,17 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             }
         }
     } else if (warp == 1 && leader && lane == 0) {
-        // ====================== MMA issuer: one thread for both CTAs of the pair ======================
+        // ============ score MMA issuer: one thread for both CTAs of the pair (S = Q K^T) ============
+        // Two issuing threads, this one and the P V issuer in warp 7: a single thread has nothing to hide the latency of
+        // its own barrier tests, commits and MMA issue behind, and the tensor pipe idled between its groups.
         constexpr uint32_t kIdescQK = idesc_bf16(128, 128, false, false);
-        constexpr uint32_t kIdescPV = idesc_bf16(128, 256, false, true);
         constexpr uint32_t kHi = desc_hi_sw128(1024);
-        const uint32_t q_lo = desc_lo_sw128(sQ, 16), k_lo = desc_lo_sw128(sK, 16), p_lo = desc_lo_sw128(sP, 16);
-        const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
-        const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
-        uint32_t q_it = 0, kc = 0, vc = 0, tc = 0, vfix_it = 0, item_it = 0;
+        const uint32_t q_lo = desc_lo_sw128(sQ, 16), k_lo = desc_lo_sw128(sK, 16);
+        uint32_t q_it = 0, kc = 0, item_it = 0;   // kc: score tiles issued so far (all items)
         bool ok = true;
-        // scores of K group g (kKG slabs) into tS; the group goes back to the producer when its MMAs are done and
-        // the last group's commit also tells the softmax warps that the scores are complete
-        // The issuing thread has nothing to hide instruction latency behind, so the groups are unrolled completely with
-        // compile-time offsets: every descriptor is (a loop-invariant base) + (a constant).
+        // Scores of K group g (kKG slabs), unrolled completely with compile-time offsets: every descriptor is a
+        // loop-invariant base plus a constant.  The group goes back to the producer when its MMAs are done; the last
+        // group's commit also tells the softmax warps that the scores are complete.
         auto qk_group_c = [&](auto gc, uint32_t tS, uint32_t bar_last) {
             constexpr int g = decltype(gc)::value;
 #pragma unroll
@@ -433,12 +432,46 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             }
             tc_commit2(g < kKGroups - 1 ? bar_k_empty + 8 * g : bar_last, 3);
         };
-        auto qk_group = [&](uint32_t tS, int g, uint32_t bar_last) {
-            static_assert(kKGroups == 3, "one case per K group");
-            if (g == 0) qk_group_c(std::integral_constant<int, 0>{}, tS, bar_last);
-            else if (g == 1) qk_group_c(std::integral_constant<int, 1>{}, tS, bar_last);
-            else qk_group_c(std::integral_constant<int, 2>{}, tS, bar_last);
-        };
+        static_assert(kKGroups == 3, "one call per K group");
+        for (int item = pair; item < total_items && ok; item += num_pairs) {
+            WorkUnit u;
+            int h;
+            if (!get_item(item, u, h)) continue;
+            const int n = tile_hi(u) - u.kv_begin;
+            ++item_it;
+            ok = mbar_wait(bar_q_full, q_it & 1, s_abort, 821);
+            ++q_it;
+            for (int jj = 0; jj < n && ok; ++jj) {
+                const uint32_t b = kc & 1, kpar = kc & 1;
+                const uint32_t tS = tmem_base + b * 64, bar_s = bar_s_full + 8 * b;
+                // S[b] was last read by the softmax of two tiles ago: its P is ready <=> that read is over
+                if (kc >= 2) ok = mbar_wait_cluster(bar_p_full + 8 * b, ((kc - 2) >> 1) & 1, s_abort, 820);
+                if (!ok) break;
+                VPP_TR(2, jj, 0);
+                ok = mbar_wait(bar_k_full, kpar, s_abort, 822);
+                if (!ok) break;
+                tc_fence_after();
+                qk_group_c(std::integral_constant<int, 0>{}, tS, bar_s);
+                ok = mbar_wait(bar_k_full + 8, kpar, s_abort, 822);
+                if (!ok) break;
+                tc_fence_after();
+                qk_group_c(std::integral_constant<int, 1>{}, tS, bar_s);
+                ok = mbar_wait(bar_k_full + 16, kpar, s_abort, 822);
+                if (!ok) break;
+                tc_fence_after();
+                qk_group_c(std::integral_constant<int, 2>{}, tS, bar_s);
+                ++kc;
+            }
+        }
+    } else if (warp == 7 && leader && lane == 0) {
+        // ============ P V MMA issuer: one thread for both CTAs of the pair (O += P V) ============
+        constexpr uint32_t kIdescPV = idesc_bf16(128, 256, false, true);
+        constexpr uint32_t kHi = desc_hi_sw128(1024);
+        const uint32_t p_lo = desc_lo_sw128(sP, 16);
+        const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
+        const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
+        uint32_t vc = 0, vfix_it = 0, item_it = 0;   // vc: P V tiles issued so far (all items)
+        bool ok = true;
         // O += P V for V group g: chunk c = (key half c >> 1, output half c & 1)
         auto pv_group_c = [&](auto gc, auto firstc) {
             constexpr int g = decltype(gc)::value;
@@ -454,78 +487,35 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             }
             tc_commit2(g < kVGroups - 1 ? bar_v_empty + 8 * g : bar_pv_done, 3);
         };
-        auto pv_group = [&](int g, bool first_tile) {
-            static_assert(kVGroups == 2, "one case per V group");
-            if (g == 0) {
-                if (first_tile) pv_group_c(std::integral_constant<int, 0>{}, std::true_type{});
-                else pv_group_c(std::integral_constant<int, 0>{}, std::false_type{});
-            } else {
-                if (first_tile) pv_group_c(std::integral_constant<int, 1>{}, std::true_type{});
-                else pv_group_c(std::integral_constant<int, 1>{}, std::false_type{});
-            }
-        };
+        static_assert(kVGroups == 2, "one call per V group");
         for (int item = pair; item < total_items && ok; item += num_pairs) {
             WorkUnit u;
             int h;
             if (!get_item(item, u, h)) continue;
             const int n = tile_hi(u) - u.kv_begin;
             ++item_it;
-            ok = mbar_wait(bar_q_full, q_it & 1, s_abort, 821);
-            if (!ok) break;
-            ++q_it;
-            for (int g = 0; g < kKGroups && ok; ++g) {
-                ok = mbar_wait(bar_k_full + 8 * g, kc & 1, s_abort, 822);
-                if (!ok) break;
-                tc_fence_after();
-                qk_group(tmem_base + (tc & 1) * 64, g, bar_s_full + 8 * (tc & 1));
-            }
-            if (!ok) break;
-            ++kc;
-            for (int jj = 0; jj < n; ++jj) {
+            for (int jj = 0; jj < n && ok; ++jj) {
                 const int tile0 = (u.kv_begin + jj) * kTileN;
-                const uint32_t b = tc & 1;
-                const bool tail = tile0 + kTileN > u.kv_len;
-                VPP_TR(0, jj, 0);
-                // Two streams of work: the scores of tile jj + 1 (they overlap this tile's softmax) and P V of this
-                // tile.  Whichever has its operands in shared memory is issued next, scores first.
-                const int nq = jj + 1 < n ? kKGroups : 0;
-                int qg = 0, pg = 0, spins = 0;
-                bool p_ready = false;
-                long long t0 = 0;
-                while (qg < nq || pg < kVGroups) {
-                    if (qg < nq && mbar_try_wait(bar_k_full + 8 * qg, kc & 1)) {
-                        tc_fence_after();
-                        VPP_TR(2, jj, qg);
-                        qk_group(tmem_base + (b ^ 1) * 64, qg, bar_s_full + 8 * (b ^ 1));
-                        ++qg;
-                        continue;
-                    }
-                    if (!p_ready)
-                        p_ready = mbar_try_wait_cluster(bar_p_full + 8 * b, (tc >> 1) & 1) &&
-                                  (!tail || mbar_try_wait_cluster(bar_vfix, vfix_it & 1));
-                    if (p_ready && mbar_try_wait(bar_v_full + 8 * pg, vc & 1)) {
-                        tc_fence_after();
-                        VPP_TR(3, jj, pg);
-                        pv_group(pg, jj == 0);
-                        ++pg;
-                        continue;
-                    }
-                    if ((++spins & 63) == 0) {
-                        if (t0 == 0) t0 = clock64();
-                        if (*s_abort != 0) ok = false;
-                        else if (clock64() - t0 > kWaitLimitCycles) {
-                            atomicCAS(const_cast<int*>(s_abort), 0, 826);
-                            ok = false;
-                        }
-                        if (!ok) break;
-                    }
+                const uint32_t b = vc & 1, vpar = vc & 1;
+                ok = mbar_wait_cluster(bar_p_full + 8 * b, (vc >> 1) & 1, s_abort, 826);
+                if (ok && tile0 + kTileN > u.kv_len) {
+                    ok = mbar_wait_cluster(bar_vfix, vfix_it & 1, s_abort, 825);
+                    ++vfix_it;
                 }
                 if (!ok) break;
+                VPP_TR(3, jj, 0);
+                ok = mbar_wait(bar_v_full, vpar, s_abort, 824);
+                if (!ok) break;
+                tc_fence_after();
+                if (jj == 0) pv_group_c(std::integral_constant<int, 0>{}, std::true_type{});
+                else pv_group_c(std::integral_constant<int, 0>{}, std::false_type{});
+                ok = mbar_wait(bar_v_full + 8, vpar, s_abort, 824);
+                if (!ok) break;
+                tc_fence_after();
+                if (jj == 0) pv_group_c(std::integral_constant<int, 1>{}, std::true_type{});
+                else pv_group_c(std::integral_constant<int, 1>{}, std::false_type{});
                 VPP_TR(0, jj, 5);
-                if (nq) ++kc;
-                if (tail) ++vfix_it;
                 ++vc;
-                ++tc;
             }
         }
     } else if (warp >= 2 && warp <= 5) {
