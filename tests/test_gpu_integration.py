@@ -1,0 +1,68 @@
+"""GPU integration: append then attend through the C ABI, and CUDA-graph capture of one chunk step."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_26523_b200 import api, workloads as W
+from parity import compare
+
+pytestmark = pytest.mark.gpu
+
+
+def test_append_then_attend_matches_the_oracle():
+    """The chunk's K/V rows are cut out of a complete cache, the slots poisoned, vpp_kv_append writes them back and
+    vpp_chunk_attn_fwd attends over the result: same output as the oracle on the complete cache."""
+    prob_cpu = W.make_problem(4100, [700, 0, 131], [300, 129, 1], 8, 2, 128, 128, block_size=16, std=0.7)
+    prob = prob_cpu.to("cuda")
+    bs = 16
+    rows_k, rows_v = [], []
+    for r in range(3):
+        P, C = int(prob_cpu.prefix_len[r]), int(prob_cpu.chunk_len[r])
+        for pos in range(P, P + C):
+            blk, slot = int(prob_cpu.block_table[r, pos // bs]), pos % bs
+            rows_k.append(prob.k_cache[blk, slot].clone())
+            rows_v.append(prob.v_cache[blk, slot].clone())
+            prob.k_cache[blk, slot] = float("nan")
+            prob.v_cache[blk, slot] = float("nan")
+    k_new, v_new = torch.stack(rows_k), torch.stack(rows_v)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.vpp_kv_append(k_new, v_new, prob.k_cache, prob.v_cache, prob.block_table, prob.prefix_len, prob.chunk_len, bs,
+                      prob.max_seq_len, status=status)
+    runner = api.ChunkAttn(prob)
+    out, lse = runner.run()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and int(runner.status.item()) == 0
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(compare(out, lse, prob_cpu, rows, "append + attend"))
+
+
+@pytest.mark.parametrize("splits", [0, 3])
+def test_one_chunk_step_replays_from_a_cuda_graph(splits):
+    """Work decomposition + attention (+ merge) enqueue only stream work, so a call can be captured once and replayed
+    with new contents in the same buffers."""
+    prob = W.make_problem(4200, [500, 64], [200, 1], 4, 2, 128, 128, block_size=16, std=0.7).to("cuda")
+    runner = api.ChunkAttn(prob, num_kv_splits=splits)
+    runner.run()                                  # first call outside capture (module / attribute set-up)
+    torch.cuda.synchronize()
+    eager = runner.out.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        side.wait_stream(torch.cuda.current_stream())
+        graph.capture_begin()
+        runner.run(side.cuda_stream)
+        graph.capture_end()
+    runner.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(runner.out.view(torch.int16), eager.view(torch.int16))
+    # new queries in the same buffer: the replay recomputes
+    prob.q.mul_(-1.0)
+    graph.replay()
+    torch.cuda.synchronize()
+    runner2_out = runner.out.clone()
+    runner.run()
+    torch.cuda.synchronize()
+    assert torch.equal(runner.out.view(torch.int16), runner2_out.view(torch.int16))
+    assert not torch.equal(runner2_out.view(torch.int16), eager.view(torch.int16))
