@@ -273,3 +273,57 @@ def cfg5(device="cpu", scale_lengths=1.0):
         P = [int(p * scale_lengths) for p in P]
     return make_problem(BASE_SEED + 5, P, C, 64, 8, 128, 128, block_size=128, device=device,
                         name="cfg5")
+
+
+# ----------------------------------------------------------------------------------------------
+# Index lists for index-selected (sparse) attention over the latent cache
+# ----------------------------------------------------------------------------------------------
+
+def make_sparse_indices(seed, prefix_lens, chunk_lens, topk, kind="scattered", window=None, group=64, pool_factor=1.5,
+                        pad=-1):
+    """Per-token lists of selected key positions, int32 [total_q, topk] (numpy), seeded.
+
+    Stands in for the output of a learned top-k indexer (the paper's MLA + DSA model; no trained weights here).  Every
+    list holds distinct causal positions (<= the token's own position); a token with fewer than topk causal positions
+    lists them all and pads with `pad`.  The order inside a list is shuffled.
+      kind="scattered": the `window` most recent positions (default topk/4) plus uniformly random earlier positions --
+                        no two tokens share more than chance: the worst case for cache reuse.
+      kind="clustered": the same window, and the earlier positions of all tokens of a group of `group` consecutive
+                        tokens are drawn from one pool of pool_factor * topk random positions -- neighbouring tokens
+                        select mostly the same keys, as a trained indexer's lists do.
+    """
+    rng = np.random.default_rng(int(seed))
+    total = int(sum(chunk_lens))
+    out = np.full((total, topk), pad, dtype=np.int32)
+    window = topk // 4 if window is None else int(window)
+    row = 0
+    for P, C in zip(prefix_lens, chunk_lens):
+        for g0 in range(0, C, group):
+            g1 = min(C, g0 + group)
+            lo_pos = P + g0                       # every token of the group may see positions <= lo_pos
+            pool = None
+            if kind == "clustered" and lo_pos + 1 > topk:
+                n_pool = min(lo_pos + 1, int(pool_factor * topk))
+                pool = rng.choice(lo_pos + 1, size=n_pool, replace=False)
+            for i in range(g0, g1):
+                pos = P + i
+                if pos + 1 <= topk:
+                    sel = np.arange(pos + 1)
+                else:
+                    recent = np.arange(pos + 1 - window, pos + 1)
+                    n_far = topk - window
+                    if pool is not None:
+                        cand = pool[pool < pos + 1 - window]
+                        far = cand[rng.permutation(cand.size)[:n_far]]
+                    else:
+                        far = np.empty(0, np.int64)
+                    if far.size < n_far:          # top up with uniform picks outside what is already chosen
+                        need = n_far - far.size
+                        extra = rng.choice(pos + 1 - window, size=min(pos + 1 - window, need + far.size), replace=False)
+                        extra = extra[~np.isin(extra, far)][:need]
+                        far = np.concatenate([far, extra])
+                    sel = np.concatenate([recent, far])
+                sel = sel[rng.permutation(sel.size)]
+                out[row + i, : sel.size] = sel
+        row += C
+    return out
