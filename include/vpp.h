@@ -230,6 +230,59 @@ typedef struct {
 
 vpp_status vpp_kv_append(const vpp_kv_append_args *args, vpp_stream_t stream);
 
+/*
+ * Index-selected (sparse) chunk attention over the absorbed-MLA latent cache: the attention of the paper's third
+ * model ("MLA + DSA sparse attention", evaluation set-up; its "Impact of Sparse Attention" paragraph is about the
+ * flat cost curve this has).  The selection itself (a learned top-k indexer) is an input: for every query token a
+ * list of key positions of its own request, shared by all q-heads.  Eq. 1 is evaluated over the listed keys:
+ *   entry e of token t (position pos = prefix_len[r] + i) takes part iff 0 <= e <= pos; any other value is skipped;
+ *   a position listed twice counts twice; out = softmax(scale q.k_e) v_e over the entries that take part, lse = log
+ *   of the sum of their exp(scale q.k_e); a token with no entry that takes part gets out = 0 and lse = -inf.
+ *
+ * q            bf16 [total_q, num_q_heads, 576], dense, packed request-major. 16-byte aligned. num_q_heads <= 128.
+ * kv_cache     bf16 latent cache, one kv-head of 576 features per position; values are features 0..511 of the same
+ *              row.  Position pos of request r is row block_table[r][pos / block_size] * block_size + pos % block_size
+ *              (block_table NULL: r * max_seq_len + pos); rows are kv_row_stride elements apart (a multiple of 8,
+ *              >= 576), so a paged cache must have block stride = block_size * row stride.  16-byte aligned.  The
+ *              cache must hold the chunk's own positions (every token's own row is read).
+ * indices      int32 [total_q, topk], topk >= 1.
+ * block_table, prefix_len, chunk_len, num_reqs (<= 8192), max_blocks_per_req, block_size (power of two), num_blocks,
+ * total_q, max_seq_len, softmax_scale: as in vpp_chunk_attn_args.
+ * out          bf16 [total_q, num_q_heads, 512]; lse float [total_q, num_q_heads] or NULL.
+ * workspace    device memory of at least vpp_sparse_attn_workspace_size(total_q) bytes, 16-byte aligned; owned by the
+ *              caller, contents irrelevant on entry.
+ * status       optional device int32, zeroed by the call; VPP_DEV_BAD_LENGTHS (nothing is written),
+ *              VPP_DEV_BAD_BLOCK (a needed block_table entry outside [0, num_blocks): results undefined but no
+ *              access leaves the cache) or VPP_DEV_TIMEOUT as in vpp_chunk_attn_fwd.
+ * Returns after enqueueing two kernels on `stream`; no allocation, no synchronisation.
+ */
+typedef struct {
+    const void *q;
+    const void *kv_cache;
+    int64_t kv_row_stride;
+    const int32_t *indices;
+    int32_t topk;
+    const int32_t *block_table;
+    const int32_t *prefix_len;
+    const int32_t *chunk_len;
+    int32_t num_reqs;
+    int32_t max_blocks_per_req;
+    int32_t block_size;
+    int32_t num_blocks;
+    int32_t total_q;
+    int32_t max_seq_len;
+    int32_t num_q_heads;
+    float softmax_scale;
+    void *out;
+    float *lse;
+    void *workspace;
+    size_t workspace_bytes;
+    int32_t *status;
+} vpp_sparse_attn_args;
+
+size_t vpp_sparse_attn_workspace_size(int32_t total_q);
+vpp_status vpp_sparse_mla_fwd(const vpp_sparse_attn_args *args, vpp_stream_t stream);
+
 /* Static description of a status code. */
 const char *vpp_status_string(vpp_status s);
 

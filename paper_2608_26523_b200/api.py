@@ -20,7 +20,7 @@ VPP_ERR_TIMEOUT = -5
 
 EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_status_string",
            "vpp_last_error", "vpp_last_launch_count", "vpp_chunk_attn_fwd_static", "vpp_static_scratch_bytes",
-           "vpp_static_last_error", "vpp_kv_append"]
+           "vpp_static_last_error", "vpp_kv_append", "vpp_sparse_attn_workspace_size", "vpp_sparse_mla_fwd"]
 
 
 class VppError(RuntimeError):
@@ -57,6 +57,19 @@ class KvAppendArgs(ctypes.Structure):
     ]
 
 
+class SparseAttnArgs(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("kv_cache", ctypes.c_void_p), ("kv_row_stride", ctypes.c_int64),
+        ("indices", ctypes.c_void_p), ("topk", ctypes.c_int32),
+        ("block_table", ctypes.c_void_p), ("prefix_len", ctypes.c_void_p), ("chunk_len", ctypes.c_void_p),
+        ("num_reqs", ctypes.c_int32), ("max_blocks_per_req", ctypes.c_int32), ("block_size", ctypes.c_int32),
+        ("num_blocks", ctypes.c_int32), ("total_q", ctypes.c_int32), ("max_seq_len", ctypes.c_int32),
+        ("num_q_heads", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+        ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t), ("status", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -85,6 +98,10 @@ def load_library():
         lib.vpp_static_last_error.restype = ctypes.c_char_p
         lib.vpp_kv_append.restype = ctypes.c_int
         lib.vpp_kv_append.argtypes = [ctypes.POINTER(KvAppendArgs), ctypes.c_void_p]
+        lib.vpp_sparse_attn_workspace_size.restype = ctypes.c_size_t
+        lib.vpp_sparse_attn_workspace_size.argtypes = [ctypes.c_int32]
+        lib.vpp_sparse_mla_fwd.restype = ctypes.c_int
+        lib.vpp_sparse_mla_fwd.argtypes = [ctypes.POINTER(SparseAttnArgs), ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -197,6 +214,54 @@ def vpp_kv_append(k_new, v_new, k_cache, v_cache, block_table, prefix_len, chunk
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
     _check(load_library().vpp_kv_append(ctypes.byref(a), ctypes.c_void_p(stream)))
+
+
+def vpp_sparse_attn_workspace_size(total_q):
+    return int(load_library().vpp_sparse_attn_workspace_size(int(total_q)))
+
+
+def vpp_sparse_mla_fwd(args, stream=None):
+    """Enqueue index-selected attention over the latent cache for a filled-in SparseAttnArgs."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_sparse_mla_fwd(ctypes.byref(args), ctypes.c_void_p(stream)))
+
+
+class SparseAttn:
+    """Owns out / lse / workspace / status of one sparse launch over a Problem with an absorbed-MLA latent cache.
+
+    indices: int32 [total_q, topk] device tensor of key positions (see include/vpp.h)."""
+
+    def __init__(self, prob, indices, want_lse=True):
+        dev = prob.q.device
+        assert prob.head_dim_qk == 576 and prob.head_dim_v == 512 and prob.num_kv_heads == 1
+        assert indices.dtype == torch.int32 and indices.is_contiguous() and indices.shape[0] == prob.total_q
+        kc = prob.k_cache
+        assert kc.stride(3) == 1 and (prob.block_table is None or kc.stride(0) == kc.shape[1] * kc.stride(1))
+        self.prob, self.indices = prob, indices
+        self.out = torch.empty((prob.total_q, prob.num_q_heads, 512), dtype=torch.bfloat16, device=dev)
+        self.lse = torch.empty((prob.total_q, prob.num_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.workspace = torch.empty(max(vpp_sparse_attn_workspace_size(prob.total_q), 256), dtype=torch.uint8, device=dev)
+        a = SparseAttnArgs()
+        a.q, a.kv_cache, a.kv_row_stride = _ptr(prob.q), _ptr(kc), kc.stride(1)
+        a.indices, a.topk = _ptr(indices), indices.shape[1]
+        a.block_table, a.prefix_len, a.chunk_len = _ptr(prob.block_table), _ptr(prob.prefix_len), _ptr(prob.chunk_len)
+        a.num_reqs = prob.num_reqs
+        a.max_blocks_per_req = 0 if prob.block_table is None else prob.block_table.shape[1]
+        a.block_size = prob.block_size
+        a.num_blocks = kc.shape[0]
+        a.total_q = prob.total_q
+        a.max_seq_len = prob.max_seq_len if prob.block_table is not None else kc.shape[1]
+        a.num_q_heads = prob.num_q_heads
+        a.softmax_scale = prob.scale
+        a.out, a.lse, a.status = _ptr(self.out), _ptr(self.lse), _ptr(self.status)
+        a.workspace, a.workspace_bytes = _ptr(self.workspace), self.workspace.numel()
+        self.args = a
+
+    def run(self, stream=None):
+        vpp_sparse_mla_fwd(self.args, stream)
+        return self.out, self.lse
 
 
 def vpp_last_launch_count():

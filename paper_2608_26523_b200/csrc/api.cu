@@ -14,6 +14,7 @@
 #include "attn_simple.cuh"
 #include "attn_mla.cuh"
 #include "attn_mla2.cuh"
+#include "attn_dsa.cuh"
 #include "attn_ws.cuh"
 #include "common.cuh"
 #include "kv_append.cuh"
@@ -561,6 +562,103 @@ vpp_status vpp_kv_append(const vpp_kv_append_args* a, vpp_stream_t stream_) {
     vpp::kv_append_kernel<<<static_cast<unsigned>(blocks), vpp::kAppendThreads, smem, stream>>>(p);
     cudaError_t ce = cudaGetLastError();
     if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "append launch: %s", cudaGetErrorString(ce));
+    return VPP_OK;
+}
+
+size_t vpp_sparse_attn_workspace_size(int32_t total_q) {
+    return 256 + sizeof(int2) * static_cast<size_t>(total_q > 0 ? total_q : 0);
+}
+
+vpp_status vpp_sparse_mla_fwd(const vpp_sparse_attn_args* a, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    if (!a) return fail(VPP_ERR_INVALID_ARG, "args is null");
+    if (a->num_reqs < 0 || a->total_q < 0) return fail(VPP_ERR_INVALID_ARG, "num_reqs and total_q must be >= 0");
+    if (a->num_q_heads <= 0 || a->num_q_heads > 2 * vpp::kMla2Rows)
+        return fail(VPP_ERR_UNSUPPORTED, "num_q_heads must be in 1..%d", 2 * vpp::kMla2Rows);
+    if (a->topk < 1) return fail(VPP_ERR_INVALID_ARG, "topk must be >= 1");
+    if (!(a->softmax_scale > 0.f) || !std::isfinite(a->softmax_scale))
+        return fail(VPP_ERR_INVALID_ARG, "softmax_scale must be positive and finite");
+    if (a->num_reqs > vpp::kDsaMaxReqs) return fail(VPP_ERR_UNSUPPORTED, "at most %d requests", vpp::kDsaMaxReqs);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (a->status && cudaMemsetAsync(a->status, 0, sizeof(int32_t), stream) != cudaSuccess)
+        return fail(VPP_ERR_CUDA, "memset status: %s", cudaGetErrorString(cudaGetLastError()));
+    if (a->total_q == 0 || a->num_reqs == 0) return VPP_OK;
+    if (!a->q || !a->kv_cache || !a->indices || !a->prefix_len || !a->chunk_len || !a->out)
+        return fail(VPP_ERR_INVALID_ARG, "q, kv_cache, indices, prefix_len, chunk_len and out must be non-null");
+    if ((reinterpret_cast<uintptr_t>(a->q) | reinterpret_cast<uintptr_t>(a->kv_cache) | reinterpret_cast<uintptr_t>(a->out) |
+         reinterpret_cast<uintptr_t>(a->workspace)) & 15u)
+        return fail(VPP_ERR_INVALID_ARG, "q, kv_cache, out and workspace must be 16-byte aligned");
+    if (a->kv_row_stride < vpp::kMlaDqk || a->kv_row_stride % 8)
+        return fail(VPP_ERR_INVALID_ARG, "kv_row_stride must be a multiple of 8 elements and at least %d", vpp::kMlaDqk);
+    if (!a->workspace || a->workspace_bytes < vpp_sparse_attn_workspace_size(a->total_q))
+        return fail(VPP_ERR_WORKSPACE, "workspace too small: %zu bytes needed", vpp_sparse_attn_workspace_size(a->total_q));
+    int shift = 0;
+    long long capacity, num_rows;
+    if (a->block_table) {
+        if (a->block_size < 1 || (a->block_size & (a->block_size - 1)))
+            return fail(VPP_ERR_UNSUPPORTED, "block_size must be a power of two");
+        if (a->max_blocks_per_req <= 0 || a->num_blocks <= 0)
+            return fail(VPP_ERR_INVALID_ARG, "max_blocks_per_req and num_blocks must be > 0 with a block table");
+        while ((1 << shift) < a->block_size) ++shift;
+        capacity = static_cast<long long>(a->max_blocks_per_req) * a->block_size;
+        num_rows = static_cast<long long>(a->num_blocks) * a->block_size;
+    } else {
+        if (a->max_seq_len <= 0) return fail(VPP_ERR_INVALID_ARG, "max_seq_len must be > 0 for a contiguous cache");
+        capacity = a->max_seq_len;
+        num_rows = static_cast<long long>(a->num_reqs) * a->max_seq_len;
+    }
+    if (num_rows >= (1ll << 31)) return fail(VPP_ERR_UNSUPPORTED, "the cache must have fewer than 2^31 rows");
+
+    CUtensorMap tm_qh, tm_rows;
+    {
+        const uint64_t dh[4] = {64, static_cast<uint64_t>(a->num_q_heads), static_cast<uint64_t>(vpp::kMlaSlabs),
+                                static_cast<uint64_t>(a->total_q)};
+        const uint64_t sh[3] = {static_cast<uint64_t>(vpp::kMlaDqk) * 2, 128,
+                                static_cast<uint64_t>(vpp::kMlaDqk) * a->num_q_heads * 2};
+        const uint32_t bh[4] = {64, static_cast<uint32_t>(a->num_q_heads < 64 ? a->num_q_heads : 64), 1, 1};
+        // gather form: a box of one row; each copy names four rows
+        const uint64_t dr[2] = {static_cast<uint64_t>(vpp::kMlaDqk), static_cast<uint64_t>(num_rows)};
+        const uint64_t sr[1] = {static_cast<uint64_t>(a->kv_row_stride) * 2};
+        const uint32_t br[2] = {64, 1};
+        if (!make_tmap(&tm_qh, a->q, 4, dh, sh, bh) || !make_tmap(&tm_rows, a->kv_cache, 2, dr, sr, br))
+            return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(sparse mla) failed");
+    }
+    int2* tok = reinterpret_cast<int2*>(static_cast<uint8_t*>(a->workspace));
+    const int sms = sm_count_or_default();
+    {
+        long long blocks = (static_cast<long long>(a->total_q) + vpp::kDsaPrepThreads - 1) / vpp::kDsaPrepThreads;
+        if (blocks > 4ll * sms) blocks = 4ll * sms;
+        const size_t smem = sizeof(int32_t) * (static_cast<size_t>(a->num_reqs) + 1);
+        vpp::dsa_tokens_kernel<<<static_cast<unsigned>(blocks), vpp::kDsaPrepThreads, smem, stream>>>(
+            a->prefix_len, a->chunk_len, a->num_reqs, a->total_q, capacity, tok, a->status);
+        cudaError_t ce = cudaGetLastError();
+        if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "token table launch: %s", cudaGetErrorString(ce));
+    }
+    vpp::DsaParams p{};
+    p.indices = a->indices;
+    p.topk = a->topk;
+    p.tok = tok;
+    p.block_table = a->block_table;
+    p.max_blocks_per_req = a->max_blocks_per_req;
+    p.block_shift = shift;
+    p.num_blocks = a->num_blocks;
+    p.max_seq_len = a->max_seq_len;
+    p.num_q_heads = a->num_q_heads;
+    p.total_q = a->total_q;
+    p.scale_log2e = a->softmax_scale * 1.4426950408889634f;
+    p.out = a->out;
+    p.lse = a->lse;
+    p.status = a->status;
+    auto kern = vpp::dsa_attn_kernel;
+    cudaError_t ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
+    if (ce == cudaSuccess) {
+        int pairs = sms / 2;
+        if (pairs > a->total_q) pairs = a->total_q;
+        kern<<<pairs * 2, vpp::kDsaThreads, vpp::kMla2SmemBytes, stream>>>(tm_qh, tm_rows, p);
+        ce = cudaGetLastError();
+    }
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "sparse attention launch: %s", cudaGetErrorString(ce));
+    g_launches = 2;
     return VPP_OK;
 }
 

@@ -1,0 +1,115 @@
+"""GPU parity of index-selected (sparse) attention over the latent cache against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle.ref_sparse_attn import ref_sparse_chunk_attn
+from paper_2608_26523_b200 import api, workloads as W
+from parity import ABS_TOL, LSE_TOL, REL_L2_TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _bits(t):
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def _problem(seed, prefix, chunk, hq, bs=64, std=0.6):
+    return W.make_problem(seed, list(prefix), list(chunk), hq, 1, 576, 512, block_size=bs, std=std, v_aliases_k=True)
+
+
+def _check(prob_cpu, idx, tokens=None, label=""):
+    prob = prob_cpu.to("cuda")
+    runner = api.SparseAttn(prob, torch.from_numpy(idx).cuda())
+    runner.out.fill_(float("nan"))
+    runner.lse.fill_(float("nan"))
+    out, lse = runner.run()
+    torch.cuda.synchronize()
+    assert int(runner.status.item()) == 0
+    bt = None if prob_cpu.block_table is None else prob_cpu.block_table.numpy()
+    ref_o, ref_l = ref_sparse_chunk_attn(_bits(prob_cpu.q), _bits(prob_cpu.k_cache), idx, bt, prob_cpu.block_size,
+                                         prob_cpu.prefix_len.numpy(), prob_cpu.chunk_len.numpy(), 512, prob_cpu.scale, tokens)
+    sel = slice(None) if tokens is None else torch.as_tensor(tokens)
+    got_o = out.float().cpu()[sel].numpy().astype(np.float64)
+    got_l = lse.cpu()[sel].numpy().astype(np.float64)
+    assert np.isfinite(got_o).all(), label
+    err = np.abs(got_o - ref_o)
+    assert (err <= np.maximum(ABS_TOL, 2.0 ** -8 * np.abs(ref_o))).all(), "%s: max abs err %.4g" % (label, err.max())
+    rel = np.linalg.norm(got_o - ref_o) / max(np.linalg.norm(ref_o), 1e-30)
+    assert rel <= REL_L2_TOL, "%s: rel L2 %.4g" % (label, rel)
+    fin = np.isfinite(ref_l)
+    assert np.array_equal(np.isneginf(got_l), ~fin), label
+    lerr = np.abs(got_l[fin] - ref_l[fin]) / np.maximum(1.0, np.abs(ref_l[fin]))
+    assert lerr.size == 0 or lerr.max() <= LSE_TOL, "%s: lse rel err %.4g" % (label, lerr.max())
+    return dict(max_abs=float(err.max()), rel_l2=float(rel))
+
+
+@pytest.mark.parametrize("hq", [128, 64, 16, 80])
+@pytest.mark.parametrize("kind", ["scattered", "clustered"])
+def test_every_token_against_the_oracle(hq, kind):
+    # two requests, pages of 64 tokens shuffled in the pool; lists of 256 = two KV tiles; the first request starts at
+    # position 0, so its early tokens list fewer than topk positions and pad with -1
+    prefix, chunk = [0, 1500], [150, 83]
+    p = _problem(5100 + hq, prefix, chunk, hq)
+    idx = W.make_sparse_indices(61, prefix, chunk, 256, kind=kind, group=32)
+    print(_check(p, idx, label="hq%d %s" % (hq, kind)))
+
+
+@pytest.mark.parametrize("topk", [1, 100, 128, 333, 2048])
+def test_list_lengths_with_ragged_last_tile(topk):
+    prefix, chunk = [4000], [37]
+    p = _problem(5200 + topk, prefix, chunk, 128)
+    idx = W.make_sparse_indices(62 + topk, prefix, chunk, topk)
+    print(_check(p, idx, label="topk%d" % topk))
+
+
+def test_skipped_entries_duplicates_and_tokens_without_any_entry():
+    prefix, chunk = [700, 0], [70, 40]
+    p = _problem(5300, prefix, chunk, 128, bs=16)
+    rng = np.random.default_rng(8)
+    idx = W.make_sparse_indices(63, prefix, chunk, 192)
+    pos = np.concatenate([700 + np.arange(70), np.arange(40)])
+    for t in range(idx.shape[0]):
+        k = rng.integers(0, 192, size=40)
+        idx[t, k[:10]] = pos[t] + 1 + rng.integers(0, 50, size=10)     # the future
+        idx[t, k[10:20]] = -rng.integers(1, 1000, size=10)             # negative
+        idx[t, k[20:30]] = 2 ** 31 - 1 - rng.integers(0, 5, size=10)   # far outside the cache
+        idx[t, k[30:40]] = rng.integers(0, pos[t] + 1, size=10)        # duplicates of earlier positions
+    idx[5] = -1                                                        # nothing listed
+    idx[77] = pos[77] + 3                                              # only the future listed
+    idx[9, :] = -1
+    idx[9, 191] = 3                                                    # a single entry in the last slot
+    print(_check(p, idx, label="skips"))
+
+
+def test_contiguous_cache_and_wide_scores():
+    prefix, chunk = [900, 300, 0], [33, 64, 5]
+    p = W.make_problem(5400, prefix, chunk, 128, 1, 576, 512, block_size=None, std=0.7, scale=0.1, v_aliases_k=True)
+    idx = W.make_sparse_indices(64, prefix, chunk, 384, kind="clustered", group=16)
+    print(_check(p, idx, label="contiguous"))
+
+
+def test_more_tokens_than_resident_pairs_and_empty_launch():
+    prefix, chunk = [2048], [600]          # 600 tokens > 74 pairs: several tokens per pair, ragged last round
+    p = _problem(5500, prefix, chunk, 128)
+    idx = W.make_sparse_indices(65, prefix, chunk, 512, kind="clustered")
+    tokens = sorted(set(np.random.default_rng(1).integers(0, 600, size=48).tolist()) | {0, 73, 74, 147, 148, 599})
+    print(_check(p, idx, tokens=tokens, label="many tokens"))
+    # zero tokens: nothing is launched, status stays 0
+    p0 = _problem(5501, [10], [0], 128).to("cuda")
+    r0 = api.SparseAttn(p0, torch.zeros((0, 128), dtype=torch.int32, device="cuda"))
+    r0.run()
+    torch.cuda.synchronize()
+    assert int(r0.status.item()) == 0
+
+
+def test_bad_lengths_write_nothing():
+    p = _problem(5600, [100], [20], 128).to("cuda")
+    idx = torch.from_numpy(W.make_sparse_indices(66, [100], [20], 128)).cuda()
+    runner = api.SparseAttn(p, idx)
+    p.chunk_len.fill_(19)                  # does not add up to total_q
+    runner.out.fill_(7.0)
+    runner.run()
+    torch.cuda.synchronize()
+    assert int(runner.status.item()) == 1
+    assert (runner.out == 7.0).all()
