@@ -256,18 +256,90 @@ def bench_decode(args):
     return 0
 
 
+def bench_sparse(args):
+    """Index-selected (sparse) attention over the cfg3 latent cache: 8192-token chunk, Hq = 128, 2048 listed keys per
+    token, at several prefix lengths and for two list structures.  The cost per chunk should not depend on the prefix
+    (the paper's remark that sparse attention flattens the latency curve); the flop count is that of the listed keys."""
+    import torch
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    chunk, topk, hq = 8192, args.topk, 128
+    prefixes = [int(x) for x in args.prefixes.split(",")] if args.prefixes else [8192, 65536, 262144, 516096]
+    base = W.cfg3(prefix=prefixes[0], max_prefix=max(max(prefixes), args.max_prefix), device=dev)
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches = 0
+    for kind in ("clustered", "scattered"):
+        for i, pre in enumerate(prefixes):
+            q = W.random_q(W.BASE_SEED + 300 + i, chunk, hq, 576, std=0.5, device=dev)
+            prob = base.with_chunk([pre], [chunk], q)
+            idx_cpu = W.make_sparse_indices_strata(W.BASE_SEED + 400 + i, [pre], [chunk], topk, kind=kind)
+            listed = int((idx_cpu >= 0).sum())
+            idx = idx_cpu.to(dev)
+            runner = api.SparseAttn(prob, idx)
+            n = max(args.steps, 3)
+            with torch.cuda.stream(stream):
+                for _ in range(max(args.warmup, 3)):
+                    runner.run(stream.cuda_stream)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(n):
+                    runner.run(stream.cuda_stream)
+                e1.record(stream)
+            e1.synchronize()
+            assert int(runner.status.item()) == 0
+            ms = e0.elapsed_time(e1) / n
+            launches += 2 * n
+            flops = 2.0 * hq * (576 + 512) * listed
+            row_bytes = listed * 576 * 2                       # every listed row once (the value pass re-reads it on chip)
+            io_bytes = chunk * hq * (576 + 512) * 2 + idx.numel() * 4
+            rows.append({"lists": kind, "prefix": pre, "ms": round(ms, 4), "tflops": round(flops / ms / 1e9, 1),
+                         "frac_of_bf16_peak": round(flops / ms / 1e9 / peaks["bf16_tflops"], 4),
+                         "listed_rows_GB/s": round(row_bytes / ms / 1e6, 1),
+                         "frac_of_hbm_peak_if_no_reuse": round((row_bytes + io_bytes) / ms / 1e6 / peaks["hbm_gbs"], 4)})
+            del runner, idx, prob, q
+    clocks = sampler.stop()
+    top = rows[len(prefixes) - 1]          # clustered lists at the longest prefix
+    ms_all = [r["ms"] for r in rows if r["lists"] == "clustered"]
+    print(json.dumps({"metric": "sparse (index-selected) MLA chunk attention TFLOP/s over listed keys (1 B200)",
+                      "value": top["tflops"], "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step": top["ms"], "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+                      "vs_baseline": None,
+                      "config": {"workload": "sparse: cfg3 cache (Hq=128, latent 576/512, 64-token pages), chunk %d, %d listed "
+                                             "keys per token, lists = recent window of %d + stratified earlier positions "
+                                             "(clustered: shared by 64 consecutive tokens; scattered: independent)"
+                                             % (chunk, topk, topk // 4),
+                                 "l2": "the cache at the longer prefixes (75 MB - 604 MB) exceeds or fills the L2; Q and out "
+                                       "stream (2.3 GB per chunk)"},
+                      "cases": rows,
+                      "latency_flatness": {"ms_min": min(ms_all), "ms_max": max(ms_all),
+                                           "note": "clustered lists: ms per chunk across the prefixes; dense cfg3 grows "
+                                                   "2.1 us per prefix token"},
+                      "roofline": {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                   "frac": top["frac_of_bf16_peak"], "traffic": None,
+                                   "peak_source": "%s (dense bf16 matmul, burst)" % peaks["_source"],
+                                   "kernel": "dsa_attn_kernel, clustered lists, prefix %d" % top["prefix"]},
+                      "gpu_launches": launches, "clocks": clocks}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--max-prefix", type=int, default=0,
                     help="size the KV cache (and its page pool) for this prefix even if the run uses shorter ones")
+    ap.add_argument("--topk", type=int, default=2048, help="listed keys per token (--workload sparse)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -275,6 +347,8 @@ def main():
         return bench_append(args)
     if args.workload == "decode":
         return bench_decode(args)
+    if args.workload == "sparse":
+        return bench_sparse(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,

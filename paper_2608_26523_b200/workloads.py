@@ -327,3 +327,47 @@ def make_sparse_indices(seed, prefix_lens, chunk_lens, topk, kind="scattered", w
                 out[row + i, : sel.size] = sel
         row += C
     return out
+
+
+def make_sparse_indices_strata(seed, prefix_lens, chunk_lens, topk, kind="scattered", window=None, group=64):
+    """Vectorised variant of make_sparse_indices for benchmark sizes (millions of entries): int32 torch tensor
+    [total_q, topk] on the CPU.  Same structure -- the `window` most recent positions plus distinct earlier ones,
+    -1 padding when fewer than topk causal positions exist -- but the earlier positions are one uniform draw from each
+    of topk - window equal strata of [0, pos - window], which makes them distinct without rejection.
+    kind="clustered": the tokens of a group of `group` consecutive tokens use the same draws and the strata of the
+    group's first token, so their earlier selections coincide."""
+    gen = torch.Generator()
+    gen.manual_seed(int(seed))
+    window = topk // 4 if window is None else int(window)
+    n_far = topk - window
+    parts = []
+    for P, C in zip(prefix_lens, chunk_lens):
+        if C == 0:
+            continue
+        pos = P + torch.arange(C, dtype=torch.int64)                       # [C]
+        if kind == "clustered":
+            grp = torch.arange(C) // group
+            u = torch.rand((int(grp.max()) + 1, n_far), generator=gen, dtype=torch.float64)[grp]
+            span_pos = P + grp * group                                     # the group's first token
+        else:
+            u = torch.rand((C, n_far), generator=gen, dtype=torch.float64)
+            span_pos = pos
+        span = (span_pos + 1 - window).clamp(min=0).to(torch.float64)      # earlier positions available
+        k = torch.arange(n_far, dtype=torch.float64)
+        w = span[:, None] / n_far                                          # stratum k = [floor(k w), floor((k+1) w))
+        lo, hi = (k[None, :] * w).floor(), ((k[None, :] + 1) * w).floor()
+        far = (lo + (u * (hi - lo)).floor()).to(torch.int64)
+        recent = pos[:, None] - torch.arange(window, dtype=torch.int64)[None, :]
+        idx = torch.cat([recent, far], dim=1)
+        # tokens with fewer than topk causal positions (or strata narrower than one position): list 0..pos, pad with -1
+        short = (span_pos + 1 - window) < n_far
+        if short.any():
+            full = torch.arange(topk, dtype=torch.int64)[None, :].expand(int(short.sum()), topk).clone()
+            full[full > pos[short][:, None]] = -1
+            idx[short] = full
+        parts.append(idx.to(torch.int32))
+    if not parts:
+        return torch.zeros((0, topk), dtype=torch.int32)
+    out = torch.cat(parts, dim=0)
+    perm = torch.argsort(torch.rand(out.shape, generator=gen), dim=1)      # shuffle inside each list
+    return torch.gather(out, 1, perm.to(torch.int64)).contiguous()
