@@ -6,9 +6,10 @@
 // 64 per CTA of a 2-CTA cluster, exactly as in the packed single-token items of the dense pair kernel, from which the
 // MMA, softmax and barrier structure is taken.  What differs is the producer side: a KV tile is 128 listed rows that
 // lie anywhere in the cache, fetched with the gather form of the tensor copy (cp.async.bulk.tensor ... tile::gather4:
-// four rows of 64 columns per instruction, 128-byte swizzle applied on the way in).  A warp issues such copies at only
-// ~70-85 clk apiece, but warps issue independently (measured: 8 warps reach one copy per 9.4 clk per SM), so the 272
-// copies of a tile are spread over eight producer warps.  Entries that do not take part are pointed at the token's own cache row (always
+// four rows of 64 columns per instruction, 128-byte swizzle applied on the way in).  A warp issues such copies one lane
+// after the other at ~75-130 clk apiece, but warps issue independently, so the 272 copies of a tile are spread over ten
+// producer warps, two per hand-back group, each issuing one instruction per tile.  (16-byte cp.async copies by the same
+// warps were measured too: 385 TFLOP/s -- a warp keeps too few of them in flight.)  Entries that do not take part are pointed at the token's own cache row (always
 // present and finite) and masked out of the softmax through a 128-bit validity mask that the producer warp publishes
 // per tile.  The cost per token does not depend on the prefix length: the flat latency curve the paper says weakens
 // its linear-growth assumption.
@@ -19,7 +20,7 @@
 
 namespace vpp {
 
-constexpr int kDsaThreads = 448;   // 14 warps: see the role list in the kernel
+constexpr int kDsaThreads = 512;   // 16 warps: see the role list in the kernel
 constexpr int kDsaMaxReqs = 8192;
 constexpr int kDsaPrepThreads = 256;
 
@@ -106,8 +107,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDsaThreads, 1)
 dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant__ CUtensorMap tm_rows, const DsaParams p) {
     // tm_qh:   (64 cols, Hq heads, 9 slabs, T tokens) box (64, min(64, Hq), 1, 1) -- 64 q-heads of one token
     // tm_rows: (576 cols, cache rows) box (64, 1), gather mode: four listed rows of one 64-column slab per copy
-    // Per CTA, 14 warps: warps 0, 8-10 K producers (warp 0 also Q and the validity mask), warps 6, 11-13 V producers,
-    // warp 1 / warp 7 of the leader: one thread each issuing the score and the P V MMAs of the pair, warps 2-5 softmax.
+    // Per CTA, 16 warps: warps 0, 6, 8-11 K producers (two per hand-back group; warp 0 also Q and the validity masks),
+    // warps 12-15 V producers (two per group), warp 1 / warp 7 of the leader: one thread each issuing the score and
+    // the P V MMAs of the pair, warps 2-5 softmax.
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -126,6 +128,7 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
     const uint32_t bar_v_full = sBar + 312;  // [kVGroups]
     const uint32_t bar_v_empty = sBar + 344; // [kVGroups - 1]
     const uint32_t bar_mask = sBar + 376;    // [4] validity mask of a tile published (each CTA for itself)
+    const uint32_t bar_mask_free = sBar + 192;  // [4] ... and read by the four softmax warps
     uint8_t* gen_bar = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes;
     volatile int* s_abort = reinterpret_cast<volatile int*>(gen_bar + 416);
     volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(gen_bar + 420);
@@ -153,7 +156,10 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
             mbar_init(bar_v_full + 8 * i, 1);
             mbar_init(bar_v_empty + 8 * i, 1);
         }
-        for (int i = 0; i < 4; ++i) mbar_init(bar_mask + 8 * i, 1);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(bar_mask + 8 * i, 1);
+            mbar_init(bar_mask_free + 8 * i, 4);
+        }
         fence_mbar_init();
         *s_abort = 0;
         prefetch_tmap(&tm_qh);
@@ -206,35 +212,39 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
     const uint32_t pair_q_full = mapa_u32(bar_q_full, 0), pair_k_full = mapa_u32(bar_k_full, 0),
                    pair_v_full = mapa_u32(bar_v_full, 0);
 
-    if (warp == 0 || (warp >= 8 && warp <= 10)) {
+    if (warp == 0 || warp == 6 || (warp >= 8 && warp <= 11)) {
         // ===================================== Q / K producers =====================================
-        // A warp issues gather copies at ~70-85 clk apiece however many of its lanes take part, but warps issue
-        // independently: the 144 copies of a K tile are spread over four warps.  Warp wk fetches the keys
-        // 64 rank + 16 wk .. + 15 (four quads of four keys), lane = 4 * (slab within the group) + quad: 12 lanes, one
-        // copy per lane and group.  Warp 0 also loads Q and publishes the validity mask of the tile's 128 entries.
-        const int wk = warp == 0 ? 0 : warp - 7;
-        const int quad = 4 * wk + (lane & 3), sg = lane >> 2;
+        // A warp issues gather copies one lane after the other, ~75-130 clk apiece, but warps issue independently
+        // (measured: 8 warps x 16 lanes reach one copy per 13-16 clk per SM).  So every hand-back group has warps of its
+        // own and a warp issues ONE instruction per tile as soon as its group is free: K group g (slabs 3 g .. 3 g + 2 of
+        // this CTA's 64 keys = 48 copies) belongs to warps kw = 2 g and 2 g + 1, which take 8 quads of four keys each;
+        // lane = 8 * (slab within the group) + quad: 24 lanes.  Warp 0 also loads Q and publishes the validity mask of
+        // the tile's 128 entries.
+        const int kw = warp == 0 ? 0 : (warp == 6 ? 1 : warp - 6);
+        const int g = kw >> 1;
+        const int quad = 8 * (kw & 1) + (lane & 7), sg = lane >> 3;
         const int key0 = static_cast<int>(rank) * 64 + 4 * quad;          // first of this lane's four keys in the tile
-        const uint32_t dst_row = static_cast<uint32_t>(quad) * 512u;
+        const uint32_t dst = sK + (g * kKG + sg) * 8192 + static_cast<uint32_t>(quad) * 512u;
+        const int col = (g * kKG + sg) * 64;
         uint32_t kc = 0;
         bool ok = true;
         for (int t = pair; t < p.total_q && ok; t += num_pairs) {
             const int2 tk = __ldg(p.tok + t);
             if (tk.x < 0) continue;
-            // Q may be replaced once the scores of the previous item's last tile are done
             if (warp == 0) {
+                // Q may be replaced once the scores of the previous item's last tile are done
                 if (kc > 0) {
                     if (lane == 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 901);
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) break;
                 }
-                if (lane == 0) {
+                if (lane == 0 && leader) {
                     const int q_rows = p.num_q_heads < kMla2Rows ? p.num_q_heads : kMla2Rows;
-                    if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMlaSlabs * q_rows * 128);
-#pragma unroll 1
-                    for (int s = 0; s < kMlaSlabs; ++s)
-                        tma2_load_4d(sQ + s * 8192, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, s, t);
+                    mbar_arrive_expect_tx(bar_q_full, 2 * kMlaSlabs * q_rows * 128);
                 }
+                __syncwarp();
+                if (lane < kMlaSlabs)
+                    tma2_load_4d(sQ + lane * 8192, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, lane, t);
             }
             const int self_row = row_of(tk.x, tk.y);
             int e_next[4], m_next[4];
@@ -245,13 +255,15 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
 #pragma unroll
                 for (int i = 0; i < 4; ++i) e[i] = e_next[i];
                 if (warp == 0) {
-                    // validity of the tile's 128 entries: word i holds entry 4 l + i of lane l in bit l
+                    // validity of the tile's 128 entries: word i holds entry 4 l + i of lane l in bit l; a ring of four
+                    // slots that the softmax warps hand back after reading
                     uint32_t bits = 0;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) bits |= (m_next[i] >= 0 && m_next[i] <= tk.y ? 1u : 0u) << i;
                     const uint32_t w0 = __ballot_sync(0xffffffffu, bits & 1u), w1 = __ballot_sync(0xffffffffu, bits & 2u),
                                    w2 = __ballot_sync(0xffffffffu, bits & 4u), w3 = __ballot_sync(0xffffffffu, bits & 8u);
                     if (lane == 0) {
+                        if (kc >= 4) ok = mbar_wait(bar_mask_free + 8 * (kc & 3), ((kc - 4) >> 2) & 1, s_abort, 904);
                         volatile uint32_t* m = vmask + (kc & 3) * 4;
                         m[0] = w0; m[1] = w1; m[2] = w2; m[3] = w3;
                         mbar_arrive(bar_mask + 8 * (kc & 3));
@@ -260,72 +272,50 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
                 }
                 if (j + 1 < n_tiles) load_entries(t, j + 1, key0, e_next);
                 rows_of(tk.x, tk.y, self_row, e, r);
-                const uint32_t par = (kc & 1) ^ 1;
-#pragma unroll 1
-                for (int g = 0; g < kKGroups; ++g) {
-                    if (lane == 0) {
-                        if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, par, s_abort, 902);
-                        else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 902);
-                        if (ok && leader && warp == 0) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
-                    }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) break;
-                    if (sg < kKG) {
-                        const int s = g * kKG + sg;
-                        tma2_gather4(sK + s * 8192 + dst_row, &tm_rows, pair_k_full + 8 * g, s * 64, r[0], r[1], r[2], r[3]);
-                    }
+                if (lane == 0 && ok) {
+                    if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, (kc & 1) ^ 1, s_abort, 902);
+                    else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 902);
+                    if (ok && leader && (kw & 1) == 0) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                if (sg < kKG) tma2_gather4(dst, &tm_rows, pair_k_full + 8 * g, col, r[0], r[1], r[2], r[3]);
                 ++kc;
             }
         }
-    } else if (warp == 6 || warp >= 11) {
+    } else if (warp >= 12) {
         // ======================================= V producers =======================================
         // chunk c = (key half hf, instr i) holds value columns 256 i + 128 rank .. + 127 (two 64-column slabs) of keys
-        // 64 hf .. 64 hf + 63.  Group g = key half g: 64 copies, 16 per warp; warp wv fetches the quads 4 wv .. 4 wv + 3
-        // of each half, lane = 4 * (2 i + slab) + quad.
-        const int wv = warp == 6 ? 0 : warp - 10;
-        const int quad = 4 * wv + (lane & 3), s4 = lane >> 2;
-        const uint32_t dst_row = static_cast<uint32_t>(quad) * 512u;
+        // 64 hf .. 64 hf + 63.  Group hf = 64 copies = warps vw = 2 hf and 2 hf + 1 with 8 quads each,
+        // lane = 8 * (2 i + slab) + quad: all 32 lanes, one instruction per tile.
+        const int vw = warp - 12;
+        const int hf = vw >> 1;
+        const int quad = 8 * (vw & 1) + (lane & 7), s4 = lane >> 3;
+        const int key0 = hf * 64 + 4 * quad;
+        const int slab = 4 * (s4 >> 1) + 2 * static_cast<int>(rank) + (s4 & 1);
+        const uint32_t dst = sV + (2 * hf + (s4 >> 1)) * kMla2VChunk + (s4 & 1) * 8192 + static_cast<uint32_t>(quad) * 512u;
         uint32_t vc = 0;
         bool ok = true;
         for (int t = pair; t < p.total_q && ok; t += num_pairs) {
             const int2 tk = __ldg(p.tok + t);
             if (tk.x < 0) continue;
             const int self_row = row_of(tk.x, tk.y);
-            int e0_next[4], e1_next[4];
-            load_entries(t, 0, 4 * quad, e0_next);
-            load_entries(t, 0, 64 + 4 * quad, e1_next);
+            int e_next[4];
+            load_entries(t, 0, key0, e_next);
             for (int j = 0; j < n_tiles && ok; ++j) {
-                int e0[4], e1[4], r0[4], r1[4];
+                int e[4], r[4];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    e0[i] = e0_next[i];
-                    e1[i] = e1_next[i];
+                for (int i = 0; i < 4; ++i) e[i] = e_next[i];
+                if (j + 1 < n_tiles) load_entries(t, j + 1, key0, e_next);
+                rows_of(tk.x, tk.y, self_row, e, r);
+                if (lane == 0) {
+                    if (hf < kVGroups - 1) ok = mbar_wait(bar_v_empty + 8 * hf, (vc & 1) ^ 1, s_abort, 903);
+                    else if (vc > 0) ok = mbar_wait(bar_pv_done, (vc - 1) & 1, s_abort, 903);
+                    if (ok && leader && (vw & 1) == 0) mbar_arrive_expect_tx(bar_v_full + 8 * hf, 2 * kVG * kMla2VChunk);
                 }
-                if (j + 1 < n_tiles) {
-                    load_entries(t, j + 1, 4 * quad, e0_next);
-                    load_entries(t, j + 1, 64 + 4 * quad, e1_next);
-                }
-                rows_of(tk.x, tk.y, self_row, e0, r0);
-                rows_of(tk.x, tk.y, self_row, e1, r1);
-                const uint32_t par = (vc & 1) ^ 1;
-#pragma unroll 1
-                for (int g = 0; g < kVGroups; ++g) {
-                    if (lane == 0) {
-                        if (g < kVGroups - 1) ok = mbar_wait(bar_v_empty + 8 * g, par, s_abort, 903);
-                        else if (vc > 0) ok = mbar_wait(bar_pv_done, (vc - 1) & 1, s_abort, 903);
-                        if (ok && leader && warp == 6) mbar_arrive_expect_tx(bar_v_full + 8 * g, 2 * kVG * kMla2VChunk);
-                    }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) break;
-                    if (s4 < 4) {
-                        const int c = 2 * g + (s4 >> 1), sl = s4 & 1;
-                        const int slab = 4 * (s4 >> 1) + 2 * static_cast<int>(rank) + sl;
-                        const uint32_t dst = sV + c * kMla2VChunk + sl * 8192 + dst_row;
-                        if (g == 0) tma2_gather4(dst, &tm_rows, pair_v_full + 8 * g, slab * 64, r0[0], r0[1], r0[2], r0[3]);
-                        else tma2_gather4(dst, &tm_rows, pair_v_full + 8 * g, slab * 64, r1[0], r1[1], r1[2], r1[3]);
-                    }
-                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                tma2_gather4(dst, &tm_rows, pair_v_full + 8 * hf, slab * 64, r[0], r[1], r[2], r[3]);
                 ++vc;
             }
         }
@@ -454,6 +444,8 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
                 if (!ok) break;
                 const uint32_t w0 = vmask[(tc & 3) * 4], w1 = vmask[(tc & 3) * 4 + 1], w2 = vmask[(tc & 3) * 4 + 2],
                                w3 = vmask[(tc & 3) * 4 + 3];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_mask_free + 8 * (tc & 3));
                 tc_wait_ld();
                 if ((w0 & w1 & w2 & w3) != 0xffffffffu) {   // some listed entries of this tile do not take part
                     const uint32_t we[4] = {w0 >> (half * 16), w1 >> (half * 16), w2 >> (half * 16), w3 >> (half * 16)};
