@@ -113,3 +113,14 @@ def test_bad_lengths_write_nothing():
     torch.cuda.synchronize()
     assert int(runner.status.item()) == 1
     assert (runner.out == 7.0).all()
+
+
+def test_benchmark_size_launch_on_sampled_tokens():
+    """The launch bench.py times (cfg 3 cache, 8192-token chunk at prefix 65536, 2048 listed keys per token, both list
+    kinds), checked on sampled tokens that the oracle computes one by one."""
+    prob_cpu = W.cfg3(prefix=65536)
+    rng = np.random.default_rng(17)
+    tokens = sorted(set(rng.integers(0, 8192, size=20).tolist()) | {0, 1, 63, 64, 4095, 8191})
+    for kind in ("clustered", "scattered"):
+        idx = W.make_sparse_indices_strata(W.BASE_SEED + 401, [65536], [8192], 2048, kind=kind).numpy()
+        print(kind, _check(prob_cpu, idx, tokens=tokens, label="bench size " + kind))
