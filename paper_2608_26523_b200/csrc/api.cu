@@ -332,27 +332,28 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
         if (!make_tmap(&tm_k2, a->k_cache, 5, d, sk, b5) || !make_tmap(&tm_v2, a->v_cache, 5, d, sv, b5))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
     }
-    CUtensorMap tm_q9, tm_k9, tm_qh9;  // one 64-column slab of 64 rows per box
+    CUtensorMap tm_q9, tm_qh9, tm_k93, tm_k92;  // 64 rows of one 64-column slab per box (tm_k93 / tm_k92: of 3 / 2 slabs)
     const bool mla_pair = fam == Family::kMla576 && use_mla_pair_kernel(a);
     if (mla_pair) {
         const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), static_cast<uint64_t>(vpp::kMlaSlabs),
                                 static_cast<uint64_t>(a->num_q_heads)};
         const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
                                 static_cast<uint64_t>(a->head_dim_qk) * 2};
-        const uint32_t bq[4] = {64, 64, 1, 1};
+        const uint32_t bq[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // all nine slabs in one copy
         const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
                                static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
         const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
                                 static_cast<uint64_t>(a->k_block_stride) * 2};
-        const uint32_t b1[5] = {64, 64, 1, 1, 1};
-        if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) || !make_tmap(&tm_k9, a->k_cache, 5, d, sk, b1))
+        const uint32_t b3[5] = {64, 64, 3, 1, 1}, b2[5] = {64, 64, 2, 1, 1};
+        if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) ||
+            !make_tmap(&tm_k93, a->k_cache, 5, d, sk, b3) || !make_tmap(&tm_k92, a->k_cache, 5, d, sk, b2))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");
         // packed single-token items: 64 q-heads of one token as the rows of a CTA's Q tile
         const uint64_t dh[4] = {64, static_cast<uint64_t>(a->num_q_heads), static_cast<uint64_t>(vpp::kMlaSlabs),
                                 static_cast<uint64_t>(a->total_q)};
         const uint64_t sh[3] = {static_cast<uint64_t>(a->head_dim_qk) * 2, 128,
                                 static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2};
-        const uint32_t bh[4] = {64, static_cast<uint32_t>(a->num_q_heads < 64 ? a->num_q_heads : 64), 1, 1};
+        const uint32_t bh[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // heads past num_q_heads read as zero
         if (!make_tmap(&tm_qh9, a->q, 4, dh, sh, bh)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla q heads) failed");
     }
     CUtensorMap tm_k4, tm_k5;
@@ -418,7 +419,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     if (mla_pair) {
         auto kern = vpp::attn_mla2_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
-        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_k9, tm_qh9, ap);
+        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_qh9, tm_k93, tm_k92, ap);
     } else if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
@@ -615,7 +616,7 @@ vpp_status vpp_sparse_mla_fwd(const vpp_sparse_attn_args* a, vpp_stream_t stream
                                 static_cast<uint64_t>(a->total_q)};
         const uint64_t sh[3] = {static_cast<uint64_t>(vpp::kMlaDqk) * 2, 128,
                                 static_cast<uint64_t>(vpp::kMlaDqk) * a->num_q_heads * 2};
-        const uint32_t bh[4] = {64, static_cast<uint32_t>(a->num_q_heads < 64 ? a->num_q_heads : 64), 1, 1};
+        const uint32_t bh[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // heads past num_q_heads read as zero
         // gather form: a box of one row; each copy names four rows
         const uint64_t dr[2] = {static_cast<uint64_t>(vpp::kMlaDqk), static_cast<uint64_t>(num_rows)};
         const uint64_t sr[1] = {static_cast<uint64_t>(a->kv_row_stride) * 2};

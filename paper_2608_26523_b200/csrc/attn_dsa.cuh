@@ -105,7 +105,7 @@ __device__ __forceinline__ void tma2_gather4(uint32_t dst, const CUtensorMap* m,
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDsaThreads, 1)
 dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant__ CUtensorMap tm_rows, const DsaParams p) {
-    // tm_qh:   (64 cols, Hq heads, 9 slabs, T tokens) box (64, min(64, Hq), 1, 1) -- 64 q-heads of one token
+    // tm_qh:   (64 cols, Hq heads, 9 slabs, T tokens) box (64, min(64, Hq), 9, 1) -- 64 q-heads of one token, all slabs
     // tm_rows: (576 cols, cache rows) box (64, 1), gather mode: four listed rows of one 64-column slab per copy
     // Per CTA, 16 warps: warps 0, 6, 8-11 K producers (two per hand-back group; warp 0 also Q and the validity masks),
     // warps 12-15 V producers (two per group), warp 1 / warp 7 of the leader: one thread each issuing the score and
@@ -239,12 +239,9 @@ dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant
                     if (!ok) break;
                 }
                 if (lane == 0 && leader) {
-                    const int q_rows = p.num_q_heads < kMla2Rows ? p.num_q_heads : kMla2Rows;
-                    mbar_arrive_expect_tx(bar_q_full, 2 * kMlaSlabs * q_rows * 128);
+                    mbar_arrive_expect_tx(bar_q_full, 2 * kMla2QBytes);   // both CTAs' boxes, rows outside the tensor included
                 }
-                __syncwarp();
-                if (lane < kMlaSlabs)
-                    tma2_load_4d(sQ + lane * 8192, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, lane, t);
+                if (lane == 0) tma2_load_4d(sQ, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, 0, t);
             }
             const int self_row = row_of(tk.x, tk.y);
             int e_next[4], m_next[4];

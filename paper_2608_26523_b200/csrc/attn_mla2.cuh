@@ -150,12 +150,14 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMla2Threads, 1)
-attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_k1,
-                 const __grid_constant__ CUtensorMap tm_qh, const AttnParams p) {
-    // tm_qh: (64 cols, Hq heads, 9 slabs, T rows) box (64, 64, 1, 1)      -- 64 q-heads of one token (packed items)
-    // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 1, 1)         -- 64 query rows of one 64-column slab
-    // tm_k1: (64 cols, keys, 9 slabs, head, block) box (64, 64, 1, 1, 1) -- 64 keys of one 64-column slab
-    // Every tile is fetched slab by slab (8 KB copies).
+attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_qh,
+                 const __grid_constant__ CUtensorMap tm_k3, const __grid_constant__ CUtensorMap tm_k2, const AttnParams p) {
+    // tm_qh: (64 cols, Hq heads, 9 slabs, T rows) box (64, 64, 9, 1)      -- 64 q-heads of one token (packed items)
+    // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 9, 1)         -- 64 query rows, all nine 64-column slabs
+    // tm_k3: (64 cols, keys, 9 slabs, head, block) box (64, 64, 3, 1, 1) -- 64 keys of three slabs: one K hand-back group
+    // tm_k2: the same tensor, box (64, 64, 2, 1, 1)                      -- 64 keys of two slabs: one V chunk
+    // One copy per group / chunk: a thread spends 100 clk and more on every copy it issues, and the data of a group
+    // is wanted as soon as possible after its buffer is free (slab-by-slab copies: 1159 TFLOP/s on cfg 3 at 64K, this: 1234).
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -211,8 +213,9 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         fence_mbar_init();
         *s_abort = 0;
         prefetch_tmap(&tm_q1);
-        prefetch_tmap(&tm_k1);
         prefetch_tmap(&tm_qh);
+        prefetch_tmap(&tm_k3);
+        prefetch_tmap(&tm_k2);
     }
     __syncthreads();
     cluster_sync_all();  // barrier initialisation is visible to the other CTA before anything arrives remotely
@@ -301,16 +304,12 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 // Q may be replaced once the scores of the previous item's last tile are done
                 if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 801);
                 if (!ok) break;
-                // (a packed tile has min(64, Hq) rows per CTA; rows of a copy that lie outside the tensor still count)
-                const int q_rows = is_packed(u) ? (p.num_q_heads < kMla2Rows ? p.num_q_heads : kMla2Rows) : kMla2Rows;
-                if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMlaSlabs * q_rows * 128);
-#pragma unroll 1
-                for (int s = 0; s < kMlaSlabs; ++s) {
-                    if (is_packed(u))   // heads 64 rank .. 64 rank + 63 of the token (heads that do not exist read as zero)
-                        tma2_load_4d(sQ + s * 8192, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, s, u.q_row0);
-                    else
-                        tma2_load_4d(sQ + s * 8192, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, s, h);
-                }
+                if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMla2QBytes);   // both CTAs' boxes, rows outside the tensor included
+                // one copy of all nine slabs
+                if (is_packed(u))   // heads 64 rank .. 64 rank + 63 of the token (heads that do not exist read as zero)
+                    tma2_load_4d(sQ, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, 0, u.q_row0);
+                else
+                    tma2_load_4d(sQ, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, 0, h);
                 ++q_it;
                 const int t_hi = tile_hi(u);
                 int blk_next = 0, slot_next = 0;
@@ -320,16 +319,12 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                     if (j + 1 < t_hi) page_of(u, (j + 1) * kTileN + static_cast<int>(rank) * 64, blk_next, slot_next);
                     const uint32_t par = (kc & 1) ^ 1;
 #pragma unroll 1
-                    for (int s = 0; s < kMlaSlabs; ++s) {
-                        const int g = s / kKG;
-                        if (s % kKG == 0) {
-                            if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, par, s_abort, 802);
-                            else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 802);
-                            if (!ok) break;
-                            VPP_TR(3, j - u.kv_begin, 4 + s);
-                            if (leader) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
-                        }
-                        tma2_load_5d(sK + s * 8192, &tm_k1, pair_k_full + 8 * g, 0, slot_in, s, 0, blk);
+                    for (int g = 0; g < kKGroups; ++g) {
+                        if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, par, s_abort, 802);
+                        else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 802);
+                        if (!ok) break;
+                        if (leader) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
+                        tma2_load_5d(sK + g * kKG * 8192, &tm_k3, pair_k_full + 8 * g, 0, slot_in, g * kKG, 0, blk);
                     }
                     ++kc;
                 }
@@ -376,13 +371,8 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                         }
                         const int hf = c >> 1, slab0 = 4 * (c & 1) + 2 * static_cast<int>(rank);
                         const uint32_t dst = sV + c * kMla2VChunk;
-                        if (tail) {
-                            tma_load_5d(dst, &tm_k1, own_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
-                            tma_load_5d(dst + 8192, &tm_k1, own_v_full + 8 * g, 0, hf ? s1 : s0, slab0 + 1, 0, hf ? b1 : b0);
-                        } else {
-                            tma2_load_5d(dst, &tm_k1, pair_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
-                            tma2_load_5d(dst + 8192, &tm_k1, pair_v_full + 8 * g, 0, hf ? s1 : s0, slab0 + 1, 0, hf ? b1 : b0);
-                        }
+                        if (tail) tma_load_5d(dst, &tm_k2, own_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
+                        else tma2_load_5d(dst, &tm_k2, pair_v_full + 8 * g, 0, hf ? s1 : s0, slab0, 0, hf ? b1 : b0);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
