@@ -289,3 +289,68 @@ class ChunkAttn:
     def run(self, stream=None):
         vpp_chunk_attn_fwd(self.args, stream)
         return self.out, self.lse
+
+
+class HostChunkPipeline:
+    """One request's chunk whose inputs and outputs live in pinned host memory, streamed through the GPU in slices.
+
+    The chunk's query rows are cut into `slices` runs.  Slice i's query rows and the cache pages that hold its own keys
+    and values go host -> device on a copy stream; its attention (prefix = the request's prefix plus the earlier slices,
+    whose pages are in the cache by then) is enqueued on the compute stream as soon as they have landed; its output rows
+    go device -> host on a third stream.  Copies of one slice overlap the attention of its neighbours; every slice is one
+    vpp_chunk_attn_fwd call.  A step is self-contained: nothing of the next step starts before the last copy of this one."""
+
+    def __init__(self, prob, slices=4, num_kv_splits=0):
+        assert prob.num_reqs == 1 and prob.block_table is not None
+        dev = prob.q.device
+        P, C, B = int(prob.prefix_len[0]), int(prob.chunk_len[0]), prob.block_size
+        assert C % slices == 0 and (C // slices) % B == 0 and P % B == 0, "slices must cover whole cache pages"
+        self.prob, self.slices, self.step = prob, slices, C // slices
+        self.out = torch.empty((C, prob.num_q_heads, prob.head_dim_v), dtype=torch.bfloat16, device=dev)
+        self.lse = torch.empty((C, prob.num_q_heads), dtype=torch.float32, device=dev)
+        self.status = torch.zeros(slices, dtype=torch.int32, device=dev)
+        self.parts = []
+        bt = prob.block_table[0].cpu().tolist()
+        for i in range(slices):
+            lo, hi = i * self.step, (i + 1) * self.step
+            pre = torch.tensor([P + lo], dtype=torch.int32, device=dev)
+            cl = torch.tensor([hi - lo], dtype=torch.int32, device=dev)
+            a = make_args(prob.q[lo:hi], prob.k_cache, prob.v_cache, prob.block_table, pre, cl, B, prob.max_seq_len,
+                          prob.scale, num_kv_splits=num_kv_splits, out=self.out[lo:hi], lse=self.lse[lo:hi],
+                          status=self.status[i:i + 1], head_dim_v=prob.head_dim_v)
+            ws = torch.empty(max(vpp_chunk_attn_workspace_size(a), 256), dtype=torch.uint8, device=dev)
+            a.workspace, a.workspace_bytes = _ptr(ws), ws.numel()
+            blocks = [bt[j] for j in range((P + lo) // B, (P + hi) // B)]
+            self.parts.append((lo, hi, a, ws, pre, cl, blocks))
+        self.s_in, self.s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.ev_in = [torch.cuda.Event() for _ in range(slices)]
+        self.ev_done = [torch.cuda.Event() for _ in range(slices)]
+        self.ev_start, self.ev_end = torch.cuda.Event(), torch.cuda.Event()
+
+    def chunk_blocks(self):
+        """Physical cache blocks of the chunk's own positions, in order."""
+        return [b for part in self.parts for b in part[6]]
+
+    def run(self, q_host, k_pages_host, v_pages_host, out_host, lse_host, stream):
+        """q_host [C, Hq, Dqk], k_pages_host / v_pages_host: dicts block -> pinned page tensors, out_host / lse_host pinned.
+        `stream` (a torch.cuda.Stream) is the compute stream; on return it waits for the last device -> host copy."""
+        p = self.prob
+        self.ev_start.record(stream)
+        self.s_in.wait_event(self.ev_start)
+        self.s_out.wait_event(self.ev_start)
+        for i, (lo, hi, a, _ws, _pre, _cl, blocks) in enumerate(self.parts):
+            with torch.cuda.stream(self.s_in):
+                p.q[lo:hi].copy_(q_host[lo:hi], non_blocking=True)
+                for b in blocks:
+                    p.k_cache[b].copy_(k_pages_host[b], non_blocking=True)
+                    p.v_cache[b].copy_(v_pages_host[b], non_blocking=True)
+                self.ev_in[i].record(self.s_in)
+            stream.wait_event(self.ev_in[i])
+            vpp_chunk_attn_fwd(a, stream.cuda_stream)
+            self.ev_done[i].record(stream)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(self.ev_done[i])
+                out_host[lo:hi].copy_(self.out[lo:hi], non_blocking=True)
+                lse_host[lo:hi].copy_(self.lse[lo:hi], non_blocking=True)
+        self.ev_end.record(self.s_out)
+        stream.wait_event(self.ev_end)

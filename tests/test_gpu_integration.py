@@ -66,3 +66,30 @@ def test_one_chunk_step_replays_from_a_cuda_graph(splits):
     torch.cuda.synchronize()
     assert torch.equal(runner.out.view(torch.int16), runner2_out.view(torch.int16))
     assert not torch.equal(runner2_out.view(torch.int16), eager.view(torch.int16))
+
+
+def test_host_streaming_pipeline_matches_the_oracle():
+    """A chunk streamed from pinned host memory in four slices (copies overlapping attention) gives the oracle's rows."""
+    prob_cpu = W.make_problem(4300, [256], [512], 8, 2, 128, 128, block_size=64, std=0.7)
+    prob = prob_cpu.to("cuda")
+    pipe = api.HostChunkPipeline(prob, slices=4)
+    q_host = prob_cpu.q.clone().pin_memory()
+    blocks = pipe.chunk_blocks()
+    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
+    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
+    # what the pipeline has to bring in is not on the device beforehand
+    prob.q.fill_(float("nan"))
+    for b in blocks:
+        prob.k_cache[b] = float("nan")
+        prob.v_cache[b] = float("nan")
+    out_host = torch.empty((512, 8, 128), dtype=torch.bfloat16).pin_memory()
+    lse_host = torch.empty((512, 8), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    for _ in range(2):                       # a second step reuses every buffer and event
+        out_host.fill_(float("nan"))
+        pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+        stream.synchronize()
+        assert int(pipe.status.max().item()) == 0
+        rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+        print(compare(out_host, lse_host, prob_cpu, rows, "host pipeline"))
