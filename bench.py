@@ -555,7 +555,7 @@ def main():
     ach = flops_pt[i_top] / (per_pt_ms[i_top] * 1e-3) / 1e12
     # DRAM bytes of that launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of the same command
     # restricted to the prefix: profiles/attn128_ws_cfg2.md; only known for the cfg2 / 131072 launch
-    traffic = 1695.0e6 if (args.workload == "cfg2" and prefixes[i_top] == 131072) else None
+    traffic = 1708.1e6 if (args.workload == "cfg2" and prefixes[i_top] == 131072) else None
     roofline = {"bound": "tensor", "achieved": round(ach, 2), "peak": burst, "unit": "TFLOP/s",
                 "frac": round(ach / burst, 4), "traffic": traffic, "peak_source": "%s (burst bf16 matmul)" % peaks["_source"],
                 "frac_of_sustained": round(ach / sustained, 4), "kernel": "attention kernel, prefix %d" % prefixes[i_top]}
