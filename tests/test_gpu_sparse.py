@@ -124,3 +124,23 @@ def test_benchmark_size_launch_on_sampled_tokens():
     for kind in ("clustered", "scattered"):
         idx = W.make_sparse_indices_strata(W.BASE_SEED + 401, [65536], [8192], 2048, kind=kind).numpy()
         print(kind, _check(prob_cpu, idx, tokens=tokens, label="bench size " + kind))
+
+
+@pytest.mark.parametrize("seed", list(range(10)))
+def test_seeded_random_shapes(seed):
+    """Odd head counts, list lengths, page sizes and request mixes: the tile counts, ragged tiles and barrier phases
+    they produce are not the ones the hand-picked cases have."""
+    rng = np.random.default_rng(9000 + seed)
+    hq = int(rng.choice([1, 3, 8, 17, 40, 64, 65, 100, 127, 128]))
+    topk = int(rng.integers(1, 700))
+    n_req = int(rng.integers(1, 5))
+    prefix = [int(rng.integers(0, 3000)) for _ in range(n_req)]
+    chunk = [int(rng.integers(0, 90)) for _ in range(n_req)]
+    if sum(chunk) == 0:
+        chunk[0] = 5
+    bs = [None, 16, 32, 64, 128][int(rng.integers(0, 5))]
+    p = W.make_problem(9100 + seed, prefix, chunk, hq, 1, 576, 512, block_size=bs, std=0.6, v_aliases_k=True)
+    idx = W.make_sparse_indices(9200 + seed, prefix, chunk, topk, kind=["scattered", "clustered"][seed & 1], group=16)
+    holes = rng.random(idx.shape) < 0.05                      # knock out 5 % of the entries
+    idx[holes] = -1
+    print(dict(hq=hq, topk=topk, prefix=prefix, chunk=chunk, bs=bs), _check(p, idx, label="random %d" % seed))
