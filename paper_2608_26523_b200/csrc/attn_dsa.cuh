@@ -9,10 +9,10 @@
 // four rows of 64 columns per instruction, 128-byte swizzle applied on the way in).  A warp issues such copies one lane
 // after the other at ~75-130 clk apiece, but warps issue independently, so the 272 copies of a tile are spread over ten
 // producer warps, two per hand-back group, each issuing one instruction per tile.  (16-byte cp.async copies by the same
-// warps were measured too: 385 TFLOP/s -- a warp keeps too few of them in flight.)  Entries that do not take part are pointed at the token's own cache row (always
-// present and finite) and masked out of the softmax through a 128-bit validity mask that the producer warp publishes
-// per tile.  The cost per token does not depend on the prefix length: the flat latency curve the paper says weakens
-// its linear-growth assumption.
+// warps were measured too: 385 TFLOP/s -- a warp keeps too few of them in flight.)
+// Entries that do not take part are pointed at the token's own cache row (always present and finite) and masked out
+// of the softmax through a 128-bit validity mask that warp 0 publishes per tile.  The cost per token does not depend on
+// the prefix length: the flat latency curve the paper says weakens its linear-growth assumption.
 #pragma once
 #include <type_traits>
 
@@ -105,7 +105,7 @@ __device__ __forceinline__ void tma2_gather4(uint32_t dst, const CUtensorMap* m,
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kDsaThreads, 1)
 dsa_attn_kernel(const __grid_constant__ CUtensorMap tm_qh, const __grid_constant__ CUtensorMap tm_rows, const DsaParams p) {
-    // tm_qh:   (64 cols, Hq heads, 9 slabs, T tokens) box (64, min(64, Hq), 9, 1) -- 64 q-heads of one token, all slabs
+    // tm_qh:   (64 cols, Hq heads, 9 slabs, T tokens) box (64, 64, 9, 1) -- 64 q-heads of one token, all slabs (heads past Hq read as zero)
     // tm_rows: (576 cols, cache rows) box (64, 1), gather mode: four listed rows of one 64-column slab per copy
     // Per CTA, 16 warps: warps 0, 6, 8-11 K producers (two per hand-back group; warp 0 also Q and the validity masks),
     // warps 12-15 V producers (two per group), warp 1 / warp 7 of the leader: one thread each issuing the score and
