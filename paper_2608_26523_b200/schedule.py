@@ -8,7 +8,7 @@
   packing    VPP-Async over a stream of requests: the leading chunks of the next request run in the drain window
              of the current one
 
-It is fed with per-chunk latencies, either the paper's model tau_k = (k + 1) t (Eq. 1) or the latency curve that
+It is fed with per-chunk latencies, either the paper's model tau_k = (k + 1) t (Eq. 2) or the latency curve that
 bench.py measures for the attention kernel on this GPU (T(P) = a + b P per layer plus a fixed per-layer cost), and
 reports makespan, per-rank idle time and the bubble ratio.  Nothing here runs on the GPU and nothing here is on the
 attention hot path; it answers "what would the measured cost curve do to the layouts of the paper".
@@ -38,7 +38,7 @@ class Result:
 
 
 def linear_tau(t: float) -> Callable[[int], float]:
-    """Eq. 1: per-stage latency of chunk k."""
+    """Eq. 2: per-stage latency of chunk k."""
     return lambda k: (k + 1) * t
 
 
@@ -263,7 +263,7 @@ def simulate_packing(chunks: Sequence[int], tau: Callable[[int], float], comm: f
 
 
 def eq3_residual(tau: Callable[[int], float], k: int) -> float:
-    """|tau_{k-1} + tau_{k+1} - 2 tau_k| / (2 tau_k): zero when the latency is affine in k (Eq. 2)."""
+    """|tau_{k-1} + tau_{k+1} - 2 tau_k| / (2 tau_k): zero when the latency is affine in k (Eq. 3 holds exactly for the model of Eq. 2)."""
     return abs(tau(k - 1) + tau(k + 1) - 2.0 * tau(k)) / (2.0 * tau(k))
 
 

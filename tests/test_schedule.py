@@ -1,5 +1,5 @@
 """Host logic: the pipeline-layout simulator against what the paper's latency model fixes in closed form
-(tau_k = (k + 1) t, Eq. 1; tau_{k-1} + tau_{k+1} = 2 tau_k, Eq. 2; drain bubble about (N + 1) t, §3.3)."""
+(tau_k = (k + 1) t, Eq. 2; tau_{k-1} + tau_{k+1} = 2 tau_k, Eq. 3; drain bubble about (N + 1) t, the pipelined-packing section)."""
 import json
 import subprocess
 import sys
@@ -43,7 +43,7 @@ def test_cpp_closed_form(n):
 @pytest.mark.parametrize("kind", ["vpp", "vpp_async"])
 @pytest.mark.parametrize("n", [1, 2, 3, 5, 8, 16])
 def test_vpp_closed_form_and_drain_bubble(kind, n):
-    # rank 1 works without a gap from t on (Eq. 2: exit of k-1 plus entry of k+1 on rank 0 = the two middle stages
+    # rank 1 works without a gap from t on (Eq. 3: exit of k-1 plus entry of k+1 on rank 0 = the two middle stages
     # of k on rank 1), then rank 0 runs the last exit: t + n (n + 1) t + n t; each rank idles (n + 1) t in total
     r = S.simulate(kind, n, S.linear_tau(T))
     assert r.makespan == pytest.approx(T + n * (n + 1) * T + n * T)
