@@ -208,7 +208,10 @@ def bench_decode(args):
              ("16 decode rows (context 32768) + one 8192-token chunk at prefix 32768, Hq=64 Hkv=4", [32768] * 17,
               [1] * 16 + [8192], 64, 4, 128),
              ("64 decode rows, context 32768, absorbed MLA Hq=128 (576/512), 64-token pages", [32768] * 64, [1] * 64, 128, 1, 576),
-             ("256 decode rows, context 8192, absorbed MLA Hq=128 (576/512), 64-token pages", [8192] * 256, [1] * 256, 128, 1, 576)]
+             ("256 decode rows, context 8192, absorbed MLA Hq=128 (576/512), 64-token pages", [8192] * 256, [1] * 256, 128, 1, 576),
+             ("32 decode rows, context 8192, Hq=64 Hkv=8 d=128 (1 GB of K/V: the profiler-sized case)", [8192] * 32, [1] * 32, 64, 8, 128)]
+    if args.case >= 0:
+        cases = [cases[args.case]]
     stream = torch.cuda.Stream()
     rows = []
     sampler = ClockSampler(0)
@@ -340,6 +343,7 @@ def main():
     ap.add_argument("--max-prefix", type=int, default=0,
                     help="size the KV cache (and its page pool) for this prefix even if the run uses shorter ones")
     ap.add_argument("--topk", type=int, default=2048, help="listed keys per token (--workload sparse)")
+    ap.add_argument("--case", type=int, default=-1, help="run only this case of --workload decode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-slices", type=int, default=4, help="slices the end-to-end leg streams the chunk in")
