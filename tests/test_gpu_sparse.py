@@ -144,3 +144,32 @@ def test_seeded_random_shapes(seed):
     holes = rng.random(idx.shape) < 0.05                      # knock out 5 % of the entries
     idx[holes] = -1
     print(dict(hq=hq, topk=topk, prefix=prefix, chunk=chunk, bs=bs), _check(p, idx, label="random %d" % seed))
+
+
+def test_lists_of_every_causal_position_reproduce_the_dense_kernel():
+    """With every causal position listed (shuffled), the sparse entry point and the dense chunk-attention entry point
+    compute the same thing through entirely different data paths; both are held to the dense oracle."""
+    import oracle
+    from parity import compare
+    prefix, chunk = [700, 0], [150, 200]
+    p = _problem(5700, prefix, chunk, 128)
+    topk = 1024
+    rng = np.random.default_rng(4)
+    idx = np.full((sum(chunk), topk), -1, np.int32)
+    row = 0
+    for P, C in zip(prefix, chunk):
+        for i in range(C):
+            idx[row, : P + i + 1] = rng.permutation(P + i + 1)
+            row += 1
+    pg = p.to("cuda")
+    sp = api.SparseAttn(pg, torch.from_numpy(idx).cuda())
+    o_s, l_s = sp.run()
+    dn = api.ChunkAttn(pg)
+    o_d, l_d = dn.run()
+    torch.cuda.synchronize()
+    assert int(sp.status.item()) == 0 and int(dn.status.item()) == 0
+    rows = oracle.all_rows(p.chunk_len.numpy(), 128)
+    print(compare(o_s, l_s, p, rows, "sparse, all positions listed"))
+    print(compare(o_d, l_d, p, rows, "dense"))
+    assert (o_s.float() - o_d.float()).abs().max().item() <= 1e-2
+    assert (l_s - l_d).abs().max().item() <= 1e-4
