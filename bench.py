@@ -346,7 +346,8 @@ def main():
     ap.add_argument("--case", type=int, default=-1, help="run only this case of --workload decode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--e2e-slices", type=int, default=4, help="slices the end-to-end leg streams the chunk in")
+    ap.add_argument("--e2e-slices", default="4",
+                    help="the end-to-end leg streams the chunk in this many equal slices, or in slices of these lengths (a,b,c,...)")
     args = ap.parse_args()
     if args.workload == "append":
         return bench_append(args)
@@ -497,7 +498,8 @@ def main():
             # The public call for host-resident inputs: the chunk streamed in slices, copies of one slice
             # overlapping the attention of its neighbours (api.HostChunkPipeline); every step copies all inputs in and
             # all results out, and no step starts before the previous one's last copy has finished.
-            pipe = api.HostChunkPipeline(r.prob, slices=args.e2e_slices, num_kv_splits=args.splits)
+            e2e_slices = [int(x) for x in args.e2e_slices.split(",")]
+            pipe = api.HostChunkPipeline(r.prob, slices=e2e_slices[0] if len(e2e_slices) == 1 else e2e_slices, num_kv_splits=args.splits)
             k_pages = dict(zip(chunk_blocks, k_host))
             v_pages = dict(zip(chunk_blocks, v_host))
 
@@ -572,7 +574,7 @@ def main():
                        "h2d_bytes_per_step": int(e2e[2]), "d2h_bytes_per_step": int(e2e[3]),
                        "ms_per_step": round(e2e[1], 4),
                        "workload": "the chunk at prefix %d: q and the chunk's K/V pages host->device, out and lse device->host, "
-                                   "streamed in %d slices whose copies overlap the neighbouring slices' attention" % (e2e[4], args.e2e_slices)}
+                                   "streamed in slices (%s) whose copies overlap the neighbouring slices' attention" % (e2e[4], args.e2e_slices)}
     if not args.no_cpu_baseline and world == 1 and args.workload == "cfg2":
         prob_cpu = runners[prefixes.index(65536) if 65536 in prefixes else -1].prob.to("cpu")
         fl, dt, n, threads = oracle_sample_rate(prob_cpu, 15.0, np.random.default_rng(0))

@@ -301,18 +301,25 @@ class HostChunkPipeline:
     vpp_chunk_attn_fwd call.  A step is self-contained: nothing of the next step starts before the last copy of this one."""
 
     def __init__(self, prob, slices=4, num_kv_splits=0):
+        """slices: a count (equal slices) or a list of slice lengths in query rows (each a multiple of the page size).
+        Short first and last slices shorten what cannot overlap: the first copy in and the last copy out."""
         assert prob.num_reqs == 1 and prob.block_table is not None
         dev = prob.q.device
         P, C, B = int(prob.prefix_len[0]), int(prob.chunk_len[0]), prob.block_size
-        assert C % slices == 0 and (C // slices) % B == 0 and P % B == 0, "slices must cover whole cache pages"
-        self.prob, self.slices, self.step = prob, slices, C // slices
+        lens = [C // slices] * slices if isinstance(slices, int) else [int(x) for x in slices]
+        assert sum(lens) == C and all(n > 0 and n % B == 0 for n in lens) and P % B == 0, "slices must cover whole cache pages"
+        slices = len(lens)
+        bounds = [0]
+        for n in lens:
+            bounds.append(bounds[-1] + n)
+        self.prob, self.slices = prob, slices
         self.out = torch.empty((C, prob.num_q_heads, prob.head_dim_v), dtype=torch.bfloat16, device=dev)
         self.lse = torch.empty((C, prob.num_q_heads), dtype=torch.float32, device=dev)
         self.status = torch.zeros(slices, dtype=torch.int32, device=dev)
         self.parts = []
         bt = prob.block_table[0].cpu().tolist()
         for i in range(slices):
-            lo, hi = i * self.step, (i + 1) * self.step
+            lo, hi = bounds[i], bounds[i + 1]
             pre = torch.tensor([P + lo], dtype=torch.int32, device=dev)
             cl = torch.tensor([hi - lo], dtype=torch.int32, device=dev)
             a = make_args(prob.q[lo:hi], prob.k_cache, prob.v_cache, prob.block_table, pre, cl, B, prob.max_seq_len,
