@@ -346,8 +346,8 @@ def main():
     ap.add_argument("--case", type=int, default=-1, help="run only this case of --workload decode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--e2e-slices", default="4",
-                    help="the end-to-end leg streams the chunk in this many equal slices, or in slices of these lengths (a,b,c,...)")
+    ap.add_argument("--e2e-slices", default="auto",
+                    help="the end-to-end leg streams the chunk in slices: auto (planned), a count of equal slices, or lengths a,b,c,...")
     args = ap.parse_args()
     if args.workload == "append":
         return bench_append(args)
@@ -498,8 +498,13 @@ def main():
             # The public call for host-resident inputs: the chunk streamed in slices, copies of one slice
             # overlapping the attention of its neighbours (api.HostChunkPipeline); every step copies all inputs in and
             # all results out, and no step starts before the previous one's last copy has finished.
-            e2e_slices = [int(x) for x in args.e2e_slices.split(",")]
-            pipe = api.HostChunkPipeline(r.prob, slices=e2e_slices[0] if len(e2e_slices) == 1 else e2e_slices, num_kv_splits=args.splits)
+            if args.e2e_slices == "auto":
+                pipe = api.HostChunkPipeline(r.prob, slices="auto", num_kv_splits=args.splits)
+            else:
+                e2e_slices = [int(x) for x in args.e2e_slices.split(",")]
+                pipe = api.HostChunkPipeline(r.prob, slices=e2e_slices[0] if len(e2e_slices) == 1 else e2e_slices,
+                                             num_kv_splits=args.splits)
+            e2e_plan = [hi - lo for (lo, hi, *_rest) in pipe.parts]
             k_pages = dict(zip(chunk_blocks, k_host))
             v_pages = dict(zip(chunk_blocks, v_host))
 
@@ -574,7 +579,7 @@ def main():
                        "h2d_bytes_per_step": int(e2e[2]), "d2h_bytes_per_step": int(e2e[3]),
                        "ms_per_step": round(e2e[1], 4),
                        "workload": "the chunk at prefix %d: q and the chunk's K/V pages host->device, out and lse device->host, "
-                                   "streamed in slices (%s) whose copies overlap the neighbouring slices' attention" % (e2e[4], args.e2e_slices)}
+                                   "streamed in slices of %s query rows whose copies overlap the neighbouring slices' attention" % (e2e[4], e2e_plan)}
     if not args.no_cpu_baseline and world == 1 and args.workload == "cfg2":
         prob_cpu = runners[prefixes.index(65536) if 65536 in prefixes else -1].prob.to("cpu")
         fl, dt, n, threads = oracle_sample_rate(prob_cpu, 15.0, np.random.default_rng(0))

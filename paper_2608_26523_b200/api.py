@@ -300,12 +300,42 @@ class HostChunkPipeline:
     go device -> host on a third stream.  Copies of one slice overlap the attention of its neighbours; every slice is one
     vpp_chunk_attn_fwd call.  A step is self-contained: nothing of the next step starts before the last copy of this one."""
 
-    def __init__(self, prob, slices=4, num_kv_splits=0):
-        """slices: a count (equal slices) or a list of slice lengths in query rows (each a multiple of the page size).
-        Short first and last slices shorten what cannot overlap: the first copy in and the last copy out."""
+    @staticmethod
+    def plan_slices(prefix, chunk, block_size, num_q_heads, num_kv_heads, sm_count):
+        """Three slices (first, middle, last) of whole 128-row tiles.  What a step cannot overlap is the first copy in, the
+        last copy out and, per launch, the idle part of its last wave of work items (an item is one query tile of one
+        pair of q-heads and runs for as long as the prefix is long): pick the lengths that make the sum smallest."""
+        step = max(128, block_size)
+        tiles = chunk // step
+        if chunk % step or tiles < 3:
+            return [chunk]
+        group = num_q_heads // num_kv_heads
+        items_per_tile = (step // 128) * (num_q_heads // 2 if group % 2 == 0 else num_q_heads)
+        item_ms = (prefix + chunk / 2) / 128 * 2.0e-3                 # ~2 us per KV tile of an item
+        in_ms, out_ms = 0.038 * step / 128, 0.030 * step / 128        # copy time per tile of rows (q in, out back) at ~55 GB/s
+
+        def idle(k):
+            w = k * items_per_tile / sm_count
+            return (-(-k * items_per_tile // sm_count) - w) * item_ms
+
+        best = None
+        for a in range(1, tiles - 1):
+            for c in range(1, tiles - a):
+                b = tiles - a - c
+                cost = a * in_ms + c * out_ms + idle(a) + idle(b) + idle(c)
+                if best is None or cost < best[0]:
+                    best = (cost, [a * step, b * step, c * step])
+        return best[1]
+
+    def __init__(self, prob, slices="auto", num_kv_splits=0):
+        """slices: "auto" (plan_slices), a count (equal slices) or a list of slice lengths in query rows (each a multiple of
+        the page size)."""
         assert prob.num_reqs == 1 and prob.block_table is not None
         dev = prob.q.device
         P, C, B = int(prob.prefix_len[0]), int(prob.chunk_len[0]), prob.block_size
+        if slices == "auto":
+            slices = self.plan_slices(P, C, B, prob.num_q_heads, prob.num_kv_heads,
+                                      torch.cuda.get_device_properties(dev).multi_processor_count)
         lens = [C // slices] * slices if isinstance(slices, int) else [int(x) for x in slices]
         assert sum(lens) == C and all(n > 0 and n % B == 0 for n in lens) and P % B == 0, "slices must cover whole cache pages"
         slices = len(lens)

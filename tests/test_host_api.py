@@ -155,3 +155,12 @@ def test_flop_count_is_the_exact_causal_count():
     p = W.make_problem(7, [5, 0], [3, 2], 4, 2, 16, 8, block_size=None)
     pairs = (3 * 5 + 3 * 4 // 2) + (2 * 0 + 2 * 3 // 2)
     assert p.pairs() == pairs and p.flops() == 2 * 4 * (16 + 8) * pairs
+
+
+def test_pipeline_slice_plan_covers_the_chunk_in_whole_pages():
+    from paper_2608_26523_b200 import api
+    for prefix, chunk, bs, hq, hkv in [(65536, 8192, 128, 64, 4), (0, 8192, 128, 64, 8), (256, 512, 64, 8, 2), (4096, 1024, 256, 16, 16)]:
+        plan = api.HostChunkPipeline.plan_slices(prefix, chunk, bs, hq, hkv, 148)
+        assert sum(plan) == chunk and all(n > 0 and n % bs == 0 for n in plan)
+    # the benchmark's chunk: first and last slice close to two full waves of work items, the middle one to ten
+    assert api.HostChunkPipeline.plan_slices(65536, 8192, 128, 64, 4, 148) == [1152, 5888, 1152]
