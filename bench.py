@@ -306,6 +306,26 @@ def bench_sparse(args):
                          "frac_of_hbm_peak_if_no_reuse": round((row_bytes + io_bytes) / ms / 1e6 / peaks["hbm_gbs"], 4)})
             del runner, idx, prob, q
     clocks = sampler.stop()
+    cpu = None
+    if not args.no_cpu_baseline:
+        # the oracle as it stands on a bounded sample of the first case's tokens
+        import numpy as np
+        from oracle.ref_sparse_attn import ref_sparse_chunk_attn
+        pre = prefixes[0]
+        q = W.random_q(W.BASE_SEED + 300, chunk, hq, 576, std=0.5, device="cpu")
+        idx_cpu = W.make_sparse_indices_strata(W.BASE_SEED + 400, [pre], [chunk], topk, kind="clustered").numpy()
+        toks = list(range(0, chunk, 3))          # about 15 s of CPU work
+        bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+        k_cpu = base.k_cache.cpu()
+        bt = base.block_table.cpu().numpy()
+        t0 = time.perf_counter()
+        ref_sparse_chunk_attn(bits(q), bits(k_cpu), idx_cpu, bt, base.block_size, np.array([pre], np.int32),
+                              np.array([chunk], np.int32), 512, base.scale, toks)
+        dt = time.perf_counter() - t0
+        fl = 2.0 * hq * (576 + 512) * float((idx_cpu[toks] >= 0).sum())
+        cpu = {"value": round(fl / dt / 1e12, 6), "unit": "TFLOP/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": "%d tokens of the chunk at prefix %d, all heads (%.1f s of wall time; numpy, threads as the BLAS takes them)"
+                         % (len(toks), pre, dt)}
     top = rows[len(prefixes) - 1]          # clustered lists at the longest prefix
     ms_all = [r["ms"] for r in rows if r["lists"] == "clustered"]
     print(json.dumps({"metric": "sparse (index-selected) MLA chunk attention TFLOP/s over listed keys (1 B200)",
@@ -326,7 +346,7 @@ def bench_sparse(args):
                                    "frac": top["frac_of_bf16_peak"], "traffic": None,
                                    "peak_source": "%s (dense bf16 matmul, burst)" % peaks["_source"],
                                    "kernel": "dsa_attn_kernel, clustered lists, prefix %d" % top["prefix"]},
-                      "gpu_launches": launches, "clocks": clocks}))
+                      "cpu_baseline": cpu, "gpu_launches": launches, "clocks": clocks}))
     return 0
 
 
