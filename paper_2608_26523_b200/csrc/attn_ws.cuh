@@ -141,6 +141,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t bar_s_full = sBar + 48;       // [2]
     const uint32_t bar_p_full = sBar + 64;       // [2]
     const uint32_t bar_o_full = sBar + 80;       // [2]
+    // Two slots used alternately: the producer can fix up the V tile of the next short item before the MMA thread has
+    // looked at the barrier for this one (slot k & 1 for the k-th such tile, 24 bytes apart).
     const uint32_t bar_vfix = sBar + 96;
     const uint32_t bar_p_part = sBar + 104;      // [2] first kSplitCols key columns of P are in place (optional early hand-off)
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
@@ -169,6 +171,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         mbar_init(bar_q_full, 1);
         mbar_init(bar_q_empty, 1);
         mbar_init(bar_vfix, 1);
+        mbar_init(bar_vfix + 24, 1);
         mbar_init(bar_x1, 4);
         mbar_init(bar_x0, 4);
         for (int i = 0; i < kWsStages; ++i) {
@@ -209,7 +212,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp < 4) {
         if (warp == 0) {
             // ============================ scheduler + TMA producer ============================
-            uint32_t item_it = 0, q_it = 0, kv_it = 0;
+            uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_cnt = 0;
             while (true) {
                 int item = 0;
                 if (lane == 0) item = atomicAdd(&p.header->counter, 1);
@@ -336,7 +339,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             }
                             fence_proxy_async_smem();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_vfix);
+                            if (lane == 0) mbar_arrive(bar_vfix + 24 * (vfix_cnt & 1));
+                            ++vfix_cnt;
                         }
                         ++kv_it;
                     }
@@ -410,7 +414,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         ok = wait1(bar_kv_full + 8 * st, (idx / kWsStages) & 1, 322);
                         if (!ok) break;
                         if (tile0 + kTileN > u.kv_len) {
-                            ok = wait1(bar_vfix, vfix_it & 1, 323);
+                            ok = wait1(bar_vfix + 24 * (vfix_it & 1), (vfix_it >> 1) & 1, 323);
                             if (!ok) break;
                             ++vfix_it;
                         }
@@ -456,7 +460,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ++kv_it;
                     if (lane == 0) VPP_TR(0, jj, 0);
                     if (tile0 + kTileN > u.kv_len) {
-                        ok = wait1(bar_vfix, vfix_it & 1, 305);
+                        ok = wait1(bar_vfix + 24 * (vfix_it & 1), (vfix_it >> 1) & 1, 305);
                         if (!ok) break;
                         ++vfix_it;
                     }

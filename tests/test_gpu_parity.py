@@ -182,3 +182,16 @@ def test_bad_lengths_set_device_status_and_write_nothing():
     torch.cuda.synchronize()
     assert int(runner.status.item()) == 1
     assert (runner.out == 3.0).all()
+
+
+def test_many_short_requests_with_ragged_single_tiles():
+    """Hundreds of work items of one ragged KV tile each: consecutive fix-ups of value rows past the end of a sequence,
+    item boundaries at every tile."""
+    rng = np.random.default_rng(31)
+    n_req = 150
+    prefix = [int(rng.integers(0, 60)) for _ in range(n_req)]
+    chunk = [int(rng.integers(2, 40)) for _ in range(n_req)]
+    prob_cpu = W.make_problem(6100, prefix, chunk, 8, 2, 128, 128, block_size=128, std=0.8)
+    out, lse, _ = run_gpu(prob_cpu.to("cuda"))
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(compare(out, lse, prob_cpu, rows, "short ragged items"))
