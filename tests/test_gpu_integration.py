@@ -93,3 +93,44 @@ def test_host_streaming_pipeline_matches_the_oracle():
         assert int(pipe.status.max().item()) == 0
         rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
         print(compare(out_host, lse_host, prob_cpu, rows, "host pipeline"))
+
+
+def test_sparse_attention_after_append_and_from_a_cuda_graph():
+    """Latent rows of the chunk appended with vpp_kv_append (keys only: the values alias them), then index-selected
+    attention over the cache, captured once in a CUDA graph and replayed; checked against the sparse oracle."""
+    from oracle.ref_sparse_attn import ref_sparse_chunk_attn
+    prefix, chunk = [300, 64], [90, 3]
+    prob_cpu = W.make_problem(4400, prefix, chunk, 128, 1, 576, 512, block_size=64, std=0.6, v_aliases_k=True)
+    idx = W.make_sparse_indices(4401, prefix, chunk, 200, kind="clustered", group=16)
+    prob = prob_cpu.to("cuda")
+    rows = []
+    for r in range(2):
+        for pos in range(prefix[r], prefix[r] + chunk[r]):
+            blk, slot = int(prob_cpu.block_table[r, pos // 64]), pos % 64
+            rows.append(prob.k_cache[blk, slot].clone())
+            prob.k_cache[blk, slot] = float("nan")
+    k_new = torch.stack(rows)
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.vpp_kv_append(k_new, None, prob.k_cache, prob.v_cache, prob.block_table, prob.prefix_len, prob.chunk_len, 64,
+                      prob.max_seq_len, status=st)
+    sp = api.SparseAttn(prob, torch.from_numpy(idx).cuda())
+    sp.run()
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and int(sp.status.item()) == 0
+    eager = sp.out.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        side.wait_stream(torch.cuda.current_stream())
+        graph.capture_begin()
+        sp.run(side.cuda_stream)
+        graph.capture_end()
+    sp.out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(sp.out.view(torch.int16), eager.view(torch.int16))
+    bits = lambda t: t.view(torch.int16).numpy().view(np.uint16)
+    ref_o, ref_l = ref_sparse_chunk_attn(bits(prob_cpu.q), bits(prob_cpu.k_cache), idx, prob_cpu.block_table.numpy(), 64,
+                                         prob_cpu.prefix_len.numpy(), prob_cpu.chunk_len.numpy(), 512, prob_cpu.scale)
+    assert np.abs(sp.out.float().cpu().numpy() - ref_o).max() <= 1e-2
+    assert np.abs(sp.lse.cpu().numpy() - ref_l).max() <= 1e-4
