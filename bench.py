@@ -225,7 +225,7 @@ def bench_decode(args):
             prob = W.make_problem(W.BASE_SEED + 92, prefix, chunk, hq, 1, 576, 512, block_size=64, std=0.5,
                                   scale=1.0 / 192 ** 0.5, v_aliases_k=True, device=dev)
             kv_bytes = sum(p + c for p, c in zip(prefix, chunk)) * 576 * 2
-        runner = api.ChunkAttn(prob)
+        runner = api.ChunkAttn(prob, num_kv_splits=args.splits)
         n = max(args.steps, 5)
         with torch.cuda.stream(stream):
             for _ in range(max(args.warmup, 3)):
