@@ -169,6 +169,8 @@ vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t n
  *    process exits.
  *  - The first call on each device looks up the array's device address (a one-time set-up that is
  *    not a stream operation); make that first call before starting any stream capture.
+ *  - With num_kv_splits = 0 the library's own split choice is dropped (the launch runs unsplit) when its partials do
+ *    not fit the array.
  *  - A launch whose vpp_chunk_attn_workspace_size exceeds VPP_STATIC_SCRATCH_BYTES is refused
  *    with VPP_ERR_WORKSPACE and nothing is enqueued; vpp_static_last_error() says how much was needed.
  *    (Split-KV partials dominate: 4 * num_kv_splits * total_q * num_q_heads * (head_dim_v + 1) bytes.)

@@ -52,12 +52,18 @@ vpp_status vpp_chunk_attn_fwd_static(const vpp_chunk_attn_args* args, vpp_stream
         snprintf(g_static_err, sizeof g_static_err, "args is null");
         return VPP_ERR_INVALID_ARG;
     }
-    const size_t need = vpp_chunk_attn_workspace_size(args);
+    vpp_chunk_attn_args a = *args;
+    size_t need = vpp_chunk_attn_workspace_size(&a);
     if (need == 0) {
         snprintf(g_static_err, sizeof g_static_err, "invalid or unsupported arguments: %s", vpp_last_error());
         return VPP_ERR_INVALID_ARG;
     }
-    if (need > VPP_STATIC_SCRATCH_BYTES) {
+    if (need > VPP_STATIC_SCRATCH_BYTES && a.num_kv_splits == 0) {
+        // the split count was the library's choice (a throughput matter): an unsplit launch needs no partials
+        a.num_kv_splits = 1;
+        need = vpp_chunk_attn_workspace_size(&a);
+    }
+    if (need == 0 || need > VPP_STATIC_SCRATCH_BYTES) {
         snprintf(g_static_err, sizeof g_static_err,
                  "this launch needs %zu bytes of scratch but the built-in scratch holds %zu: use vpp_chunk_attn_fwd "
                  "with a workspace, or lower num_kv_splits / total_q",
@@ -70,7 +76,6 @@ vpp_status vpp_chunk_attn_fwd_static(const vpp_chunk_attn_args* args, vpp_stream
         snprintf(g_static_err, sizeof g_static_err, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
         return VPP_ERR_CUDA;
     }
-    vpp_chunk_attn_args a = *args;
     a.workspace = scratch;
     a.workspace_bytes = VPP_STATIC_SCRATCH_BYTES;
     const vpp_status st = vpp_chunk_attn_fwd(&a, stream);

@@ -60,3 +60,15 @@ def test_static_scratch_refuses_oversized_launch():
     assert ei.value.status == api.VPP_ERR_WORKSPACE
     torch.cuda.synchronize()
     assert (runner.out == 5.0).all()                         # nothing was enqueued
+
+
+def test_static_scratch_drops_the_library_chosen_split_when_its_partials_do_not_fit():
+    """8192 rows x 16 q-heads at a long prefix: left to itself the library splits this launch in two (3.46 waves of work
+    items otherwise), which takes 135 MB of partials; the static entry point runs it unsplit instead of refusing."""
+    prob = W.make_problem(9004, [16384], [8192], 16, 2, 128, 128, block_size=128).to("cuda")
+    auto = api.ChunkAttn(prob, num_kv_splits=0)
+    assert api.vpp_chunk_attn_workspace_size(auto.args) > api.vpp_static_scratch_bytes()
+    ref_out, ref_lse = _launch(prob, static=False, num_kv_splits=1)
+    out, lse = _launch(prob, static=True, num_kv_splits=0)
+    assert (out - ref_out).abs().max().item() <= 1e-2
+    assert ((lse - ref_lse).abs() <= 1e-5 * ref_lse.abs().clamp(min=1)).all()
