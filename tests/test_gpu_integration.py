@@ -134,3 +134,26 @@ def test_sparse_attention_after_append_and_from_a_cuda_graph():
                                          prob_cpu.prefix_len.numpy(), prob_cpu.chunk_len.numpy(), 512, prob_cpu.scale)
     assert np.abs(sp.out.float().cpu().numpy() - ref_o).max() <= 1e-2
     assert np.abs(sp.lse.cpu().numpy() - ref_l).max() <= 1e-4
+
+
+def test_host_streaming_pipeline_with_planned_slices():
+    """The default slice plan (first / middle / last slice of whole tiles) on a chunk of eight query tiles."""
+    prob_cpu = W.make_problem(4500, [512], [1024], 8, 2, 128, 128, block_size=128, std=0.7)
+    prob = prob_cpu.to("cuda")
+    pipe = api.HostChunkPipeline(prob)                      # slices="auto"
+    plan = [hi - lo for (lo, hi, *_r) in pipe.parts]
+    assert sum(plan) == 1024 and len(plan) == 3 and all(n % 128 == 0 and n > 0 for n in plan)
+    q_host = prob_cpu.q.clone().pin_memory()
+    blocks = pipe.chunk_blocks()
+    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
+    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
+    prob.q.fill_(float("nan"))
+    out_host = torch.empty((1024, 8, 128), dtype=torch.bfloat16).pin_memory()
+    lse_host = torch.empty((1024, 8), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+    stream.synchronize()
+    assert int(pipe.status.max().item()) == 0
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(plan, compare(out_host, lse_host, prob_cpu, rows, "planned slices"))

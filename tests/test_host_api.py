@@ -164,3 +164,45 @@ def test_pipeline_slice_plan_covers_the_chunk_in_whole_pages():
         assert sum(plan) == chunk and all(n > 0 and n % bs == 0 for n in plan)
     # the benchmark's chunk: first and last slice close to two full waves of work items, the middle one to ten
     assert api.HostChunkPipeline.plan_slices(65536, 8192, 128, 64, 4, 148) == [1152, 5888, 1152]
+
+
+def _fake_args(total_q, num_reqs, hq, hkv, max_seq_len, num_kv_splits):
+    """Arguments with placeholder pointers: the workspace query is pure host code and never dereferences them."""
+    a = api.ChunkAttnArgs()
+    fake = ctypes.c_void_p(1 << 20)
+    a.q = a.k_cache = a.v_cache = a.block_table = a.prefix_len = a.chunk_len = a.out = fake
+    a.k_block_stride = a.v_block_stride = 128 * hkv * 128
+    a.k_token_stride = a.v_token_stride = hkv * 128
+    a.k_head_stride = a.v_head_stride = 128
+    a.num_reqs, a.max_blocks_per_req, a.block_size, a.num_blocks = num_reqs, (max_seq_len + 127) // 128, 128, 1 << 16
+    a.total_q, a.max_seq_len = total_q, max_seq_len
+    a.num_q_heads, a.num_kv_heads, a.head_dim_qk, a.head_dim_v = hq, hkv, 128, 128
+    a.softmax_scale = 0.088
+    a.num_kv_splits = num_kv_splits
+    return a
+
+
+def _chosen_splits(total_q, num_reqs, hq, hkv, max_seq_len):
+    auto = api.vpp_chunk_attn_workspace_size(_fake_args(total_q, num_reqs, hq, hkv, max_seq_len, 0))
+    assert auto > 0
+    for s in range(1, 17):
+        if api.vpp_chunk_attn_workspace_size(_fake_args(total_q, num_reqs, hq, hkv, max_seq_len, s)) == auto:
+            return s
+    raise AssertionError("no forced split count reproduces the automatic workspace size")
+
+
+def test_split_choice_fills_whole_waves(lib):
+    """148 SMs assumed on a box without a GPU.  One request, d = 128: the split count whose equal work items leave the
+    least idle last wave, after the measured cost of splitting (the picks below are the measured optima)."""
+    if torch.cuda.is_available() and torch.cuda.get_device_properties(0).multi_processor_count != 148:
+        pytest.skip("the expectations are for 148 SMs")
+    assert _chosen_splits(8192, 1, 64, 4, 73728) == 1      # 2048 items: 13.8 waves
+    assert _chosen_splits(8192, 1, 32, 4, 73728) == 1      # 1024 items: 6.92 waves
+    assert _chosen_splits(8192, 1, 16, 2, 73728) == 2      # 512 items: 3.46 -> 6.92 waves
+    assert _chosen_splits(8192, 1, 8, 1, 73728) == 4       # 256 items: 1.73 -> 6.92 waves
+    assert _chosen_splits(4096, 1, 8, 1, 36864) == 1       # 128 items at a shorter prefix: splitting costs more than it saves
+    # decode batches: one packed item per (token, kv-head)
+    assert _chosen_splits(64, 64, 64, 8, 32769) == 2       # 512 items
+    assert _chosen_splits(64, 64, 64, 4, 32769) == 4       # 256 items
+    assert _chosen_splits(256, 256, 64, 8, 8193) == 1      # 2048 items
+    assert _chosen_splits(32, 32, 64, 8, 8193) == 1        # 256 short items: the start-up of more units outweighs the wave
