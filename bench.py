@@ -8,10 +8,11 @@ one batch of synthetic input: the GQA long-context chunk (64 q-heads, 4 kv-heads
 count); the per-prefix latency / TFLOP/s curve -- the cost curve the paper's V-shaped layout is built
 around -- is reported beside it in "curve".
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload ...]
 
 One JSON line on stdout (rank 0).  With --impl reference the CPU oracle is timed on the host cores on a
-bounded sample of the same workload.
+bounded sample of the same workload.  The default run (one GPU) also times the other four benchmark
+configurations, each with its own clock sample and oracle baseline, and reports them under "configs".
 """
 import argparse
 import json
@@ -103,17 +104,20 @@ class ClockSampler:
 
 
 def oracle_sample_rate(prob_cpu, target_seconds, rng):
-    """Time the fp64 oracle (as it stands) on random (row, head) samples of the workload.
+    """Time the fp64 oracle (as it stands) on random (request, row, head) samples of the workload.
 
     Returns (flops done, seconds, rows, threads)."""
     import oracle
-    C = int(prob_cpu.chunk_len[0]); P = int(prob_cpu.prefix_len[0])
+    c = prob_cpu.chunk_len.numpy().astype(np.int64)
+    pre = prob_cpu.prefix_len.numpy().astype(np.int64)
+    req_of_row = np.repeat(np.arange(len(c)), c)             # packed row -> request
+    row_in_req = np.concatenate([np.arange(x) for x in c]) if len(c) else np.zeros(0, np.int64)
     hq = prob_cpu.num_q_heads
     per_row = 2.0 * (prob_cpu.head_dim_qk + prob_cpu.head_dim_v)
 
     def run(n):
-        rows = np.stack([np.zeros(n, np.int32), rng.integers(0, C, n).astype(np.int32),
-                         rng.integers(0, hq, n).astype(np.int32)], axis=1)
+        pick = rng.integers(0, len(req_of_row), n)
+        rows = np.stack([req_of_row[pick], row_in_req[pick], rng.integers(0, hq, n)], axis=1).astype(np.int32)
         t0 = time.perf_counter()
         oracle.ref_chunk_attn_rows(prob_cpu.q, prob_cpu.k_cache, prob_cpu.v_cache,
                                    prob_cpu.k_cache.stride()[:3], prob_cpu.v_cache.stride()[:3],
@@ -122,7 +126,7 @@ def oracle_sample_rate(prob_cpu, target_seconds, rng):
                                    hq, prob_cpu.num_kv_heads, prob_cpu.head_dim_qk, prob_cpu.head_dim_v,
                                    prob_cpu.scale, rows)
         dt = time.perf_counter() - t0
-        fl = float(((P + rows[:, 1].astype(np.int64) + 1) * per_row).sum())
+        fl = float(((pre[rows[:, 0]] + rows[:, 1].astype(np.int64) + 1) * per_row).sum())
         return fl, dt
 
     threads = oracle.num_threads()
@@ -130,6 +134,213 @@ def oracle_sample_rate(prob_cpu, target_seconds, rng):
     n = int(max(threads, min(4 * threads * target_seconds / max(dt, 1e-3), 200000)))
     fl, dt = run(n)
     return fl, dt, n, threads
+
+
+def cpu_baseline_entry(prob_cpu, seconds, what):
+    fl, dt, n, threads = oracle_sample_rate(prob_cpu, seconds, np.random.default_rng(0))
+    return {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%d random (row, head) pairs of %s (%.1f s of CPU time)" % (n, what, dt)}
+
+
+def read_traffic_record(name):
+    """DRAM bytes per launch of a kernel, as recorded beside its ncu summary (profiles/<name>): key = value lines."""
+    path = os.path.join(ROOT, "profiles", name)
+    rec = {}
+    if os.path.exists(path):
+        with open(path) as f:
+            for line in f:
+                if "=" in line and not line.lstrip().startswith("#"):
+                    k, v = line.split("=", 1)
+                    rec[k.strip()] = v.strip()
+    return rec
+
+
+def fit_cost_curve(prefixes, ms):
+    """The paper's linear latency model (its Eq. 2) fitted to a measured curve, and its balance identity (its Eq. 3,
+    tau(k-1) + tau(k+1) = 2 tau(k)) on the evenly spaced points of the curve."""
+    x = np.array(prefixes, dtype=np.float64); y = np.array(ms, dtype=np.float64)
+    if len(x) < 3:
+        return None
+    b, a = np.polyfit(x, y, 1)
+    r2 = 1.0 - float(((y - (a + b * x)) ** 2).sum() / max(((y - y.mean()) ** 2).sum(), 1e-30))
+    out = {"fit_ms": {"a": round(float(a), 5), "b_per_token": float(b), "r2": round(r2, 6)},
+           "fit_residual_max_rel": round(float((np.abs(y - (a + b * x)) / y).max()), 5)}
+    # every triple (i, j, k) of measured points with x_j - x_i == x_k - x_j is an instance of Eq. 3
+    res = []
+    for j in range(1, len(x) - 1):
+        for i in range(j):
+            for k in range(j + 1, len(x)):
+                if x[j] - x[i] == x[k] - x[j]:
+                    res.append(abs(y[i] + y[k] - 2 * y[j]) / (2 * y[j]))
+    if res:
+        out["eq3_residual_max"] = round(float(max(res)), 5)
+        out["eq3_triples"] = len(res)
+    return out
+
+
+def time_points(runners, stream, steps, warmup, sampler=None):
+    """warmup untimed passes over the runners, then `steps` timed ones; per-runner median ms (CUDA events on the launching
+    stream), the whole region's ms per step, launches per step and the clock record."""
+    from paper_2608_26523_b200 import api
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            for r in runners:
+                r.run(stream.cuda_stream)
+        launches = 0
+        for r in runners:
+            r.run(stream.cuda_stream)
+            launches += api.vpp_last_launch_count()
+        stream.synchronize()
+        for r in runners:
+            assert int(r.status.item()) == 0, "device status %d" % int(r.status.item())
+        if sampler is not None:
+            sampler.start()
+            time.sleep(0.25)
+        ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in runners]
+              for _ in range(steps)]
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for s_ in range(steps):
+            for i, r in enumerate(runners):
+                ev[s_][i][0].record(stream)
+                r.run(stream.cuda_stream)
+                ev[s_][i][1].record(stream)
+        t1.record(stream)
+        stream.synchronize()
+    clocks = sampler.stop() if sampler is not None else None
+    per = [statistics.median(ev[s_][i][0].elapsed_time(ev[s_][i][1]) for s_ in range(steps)) for i in range(len(runners))]
+    return per, t0.elapsed_time(t1) / steps, launches, clocks
+
+
+def sweep_other_configs(dev, peaks, steps, warmup, with_cpu):
+    """The four benchmark configurations beside cfg 2, each timed by itself (own warm-up, own clock sample)."""
+    from paper_2608_26523_b200 import api
+    burst, sustained = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    stream = torch.cuda.Stream(device=dev)
+    out = {}
+
+    def curve_of(prefixes, per_ms, flops):
+        rows = []
+        for P, ms, fl in zip(prefixes, per_ms, flops):
+            tf = fl / (ms * 1e-3) / 1e12
+            rows.append({"prefix": P, "ms": round(ms, 4), "tflops": round(tf, 2), "frac_of_burst": round(tf / burst, 4),
+                         "frac_of_sustained": round(tf / sustained, 4)})
+        return rows
+
+    plans = [("cfg3", W.cfg3, W.CFG3_PREFIXES, 8192, 0, "absorbed MLA Hq=128 (576/512), chunk 8192, 64-token pages", 65536),
+             ("cfg4", W.cfg4, [16384 * k for k in (0, 21, 42, 63)], 16384, 4,
+              "GQA Hq=64 Hkv=8 d=128, chunk 16384, 128-token pages, split-KV S=4 + merge; 4 evenly spaced points of the 16", 65536)]
+    for name, make, prefixes, chunk, splits, desc, cpu_prefix in plans:
+        base = make(prefix=max(prefixes), max_prefix=max(prefixes), device=dev)
+        runners = [api.ChunkAttn(base.with_chunk([P], [chunk], base.q), num_kv_splits=splits) for P in prefixes]
+        per, step_ms, launches, clocks = time_points(runners, stream, steps, warmup, ClockSampler(dev.index or 0))
+        flops = [r.prob.flops() for r in runners]
+        entry = {"workload": "%s: %s" % (name, desc), "num_kv_splits": splits, "steps": steps, "warmup": warmup,
+                 "curve": curve_of(prefixes, per, flops), "cost_curve": fit_cost_curve(prefixes, per),
+                 "tflops": round(sum(flops) / (step_ms * 1e-3) / 1e12, 2), "gpu_launches": launches * steps, "clocks": clocks}
+        del runners, base
+        torch.cuda.empty_cache()
+        if with_cpu:
+            small = make(prefix=cpu_prefix, device=dev).to("cpu")
+            entry["cpu_baseline"] = cpu_baseline_entry(small, 4.0, "the chunk at prefix %d" % cpu_prefix)
+            del small
+        out[name] = entry
+
+    # cfg 5: one launch
+    prob = W.cfg5(device=dev)
+    runners = [api.ChunkAttn(prob, num_kv_splits=0)]
+    per, step_ms, launches, clocks = time_points(runners, stream, max(steps, 5), warmup, ClockSampler(dev.index or 0))
+    tf = prob.flops() / (per[0] * 1e-3) / 1e12
+    kv_tokens = int((prob.prefix_len + prob.chunk_len).sum().item())
+    out["cfg5"] = {"workload": "cfg5: 32 requests, 16384 packed query tokens, lengths log-uniform 1K-256K, Hq=64 Hkv=8 d=128, "
+                               "128-token pages, one launch", "ms": round(per[0], 4), "tflops": round(tf, 2),
+                   "frac_of_burst": round(tf / burst, 4), "frac_of_sustained": round(tf / sustained, 4),
+                   "kv_tokens": kv_tokens, "gpu_launches": launches * max(steps, 5), "clocks": clocks}
+    if with_cpu:
+        out["cfg5"]["cpu_baseline"] = cpu_baseline_entry(prob.to("cpu"), 4.0, "the batch")
+    del runners, prob
+    torch.cuda.empty_cache()
+
+    # cfg 1: four launches of 512 rows against one contiguous 2048-token cache (latency-bound: no roofline claimed)
+    runners = [api.ChunkAttn(W.cfg1(k, device=dev), num_kv_splits=0) for k in range(4)]
+    per, step_ms, launches, clocks = time_points(runners, stream, max(steps, 20), max(warmup, 5), ClockSampler(dev.index or 0))
+    rows = []
+    for k, (r, ms) in enumerate(zip(runners, per)):
+        P = 512 * k
+        byts = (P + 512) * 1 * 256 * 2 + 512 * 4 * 128 * 2 * 2 + 512 * 4 * 4      # K/V read once, q in, out + lse out
+        rows.append({"prefix": P, "us": round(ms * 1e3, 2), "tflops": round(r.prob.flops() / (ms * 1e-3) / 1e12, 2),
+                     "GB/s": round(byts / ms / 1e6, 1)})
+    out["cfg1"] = {"workload": "cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache; the whole problem is "
+                               "L2-resident and 16 work items cannot fill 148 SMs: latency-bound, no roofline claimed",
+                   "curve": rows, "us_per_chunk_mean": round(step_ms * 1e3 / 4, 2), "gpu_launches": launches * max(steps, 20),
+                   "clocks": clocks}
+    if with_cpu:
+        import oracle
+        full = W.cfg1(0, device="cpu").extra["full"]
+        rows_all = oracle.all_rows(full.chunk_len.numpy(), 4)
+        t0 = time.perf_counter()
+        oracle.ref_chunk_attn_rows(full.q, full.k_cache, full.v_cache, full.k_cache.stride()[:3], full.v_cache.stride()[:3],
+                                   None, full.block_size, full.prefix_len.numpy(), full.chunk_len.numpy(), 4, 1, 128, 128,
+                                   full.scale, rows_all)
+        dt = time.perf_counter() - t0
+        out["cfg1"]["cpu_baseline"] = {"value": round(full.flops() / dt / 1e12, 6), "unit": UNIT, "cores": oracle.num_threads(),
+                                       "kind": "oracle", "sample": "all 2048 rows x 4 heads (the four chunks; %.2f s)" % dt}
+    return out
+
+
+def bench_merge(args):
+    """vpp_lse_merge against the HBM roofline: S*(4*Dv+4) bytes read + (2*Dv+4) written per (row, head), CUDA-event timed,
+    cycling through enough distinct buffers that no launch finds its inputs in the L2."""
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    cases = [("cfg4 partials: S=2, T=16384, Hq=64, Dv=128", 2, 16384, 64, 128),
+             ("cfg4 partials: S=4, T=16384, Hq=64, Dv=128", 4, 16384, 64, 128),
+             ("cfg4 partials: S=8, T=16384, Hq=64, Dv=128", 8, 16384, 64, 128),
+             ("MLA partials: S=2, T=8192, Hq=128, Dv=512", 2, 8192, 128, 512),
+             ("MLA partials: S=4, T=8192, Hq=128, Dv=512", 4, 8192, 128, 512)]
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    total_launches = 0
+    for desc, S, T, Hq, Dv in cases:
+        bytes_call = S * T * Hq * (4 * Dv + 4) + T * Hq * (2 * Dv + 4)
+        sets = max(2, int(math.ceil(400e6 / bytes_call)))
+        o_parts = [torch.randn(S, T, Hq, Dv, device=dev) for _ in range(sets)]
+        l_parts = [torch.randn(S, T, Hq, device=dev) for _ in range(sets)]
+        out = [torch.empty(T, Hq, Dv, dtype=torch.bfloat16, device=dev) for _ in range(sets)]
+        lse = [torch.empty(T, Hq, device=dev) for _ in range(sets)]
+        n = max(args.steps, 5) * sets
+        with torch.cuda.stream(stream):
+            for i in range(max(args.warmup, 3)):
+                api.vpp_lse_merge(o_parts[i % sets], l_parts[i % sets], out[i % sets], lse[i % sets], stream.cuda_stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(n):
+                api.vpp_lse_merge(o_parts[i % sets], l_parts[i % sets], out[i % sets], lse[i % sets], stream.cuda_stream)
+            e1.record(stream)
+        e1.synchronize()
+        ms = e0.elapsed_time(e1) / n
+        total_launches += n
+        rows.append({"case": desc, "us": round(ms * 1e3, 2), "GB/s": round(bytes_call / ms / 1e6, 1),
+                     "frac_of_hbm_peak": round(bytes_call / ms / 1e6 / peaks["hbm_gbs"], 4), "bytes": bytes_call,
+                     "launches_timed": n})
+        del o_parts, l_parts, out, lse
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[1]
+    print(json.dumps({"metric": "lse-merge GB/s (read + written) vs HBM peak (1 B200)", "value": top["GB/s"], "unit": "GB/s",
+                      "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": True, "dtype": "f32",
+                      "data": "synthetic", "vs_baseline": None,
+                      "config": {"workload": "merge; " + top["case"], "l2": "distinct buffers of 400 MB or more per case"},
+                      "cases": rows,
+                      "roofline": {"bound": "hbm", "achieved": top["GB/s"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": top["frac_of_hbm_peak"], "traffic": None,
+                                   "peak_source": "%s (copy bandwidth)" % peaks["_source"], "kernel": "lse_merge_kernel, " + top["case"]},
+                      "gpu_launches": total_launches, "clocks": clocks}))
+    return 0
 
 
 def bench_append(args):
@@ -356,7 +567,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse", "merge"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -366,6 +577,7 @@ def main():
     ap.add_argument("--case", type=int, default=-1, help="run only this case of --workload decode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="cfg2 only: skip the other four configurations")
     ap.add_argument("--e2e-slices", default="auto",
                     help="the end-to-end leg streams the chunk in slices: auto (planned), a count of equal slices, or lengths a,b,c,...")
     args = ap.parse_args()
@@ -375,6 +587,8 @@ def main():
         return bench_decode(args)
     if args.workload == "sparse":
         return bench_sparse(args)
+    if args.workload == "merge":
+        return bench_merge(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,
@@ -550,6 +764,14 @@ def main():
             diff = (out_host[::7].float() - r.out[::7].float().cpu()).abs().max().item()
             assert diff <= 1e-2, "streamed chunk differs from the resident launch by %g" % diff
 
+    # ---- (cfg2, one GPU) the 96K point that makes 0 / 32K / 64K / 96K / 128K evenly spaced, outside the timed step ----
+    extra_pt = None
+    if args.workload == "cfg2" and world == 1 and not args.prefixes and max_prefix >= 98304:
+        r96 = api.ChunkAttn(base.with_chunk([98304], [chunk], base.q), num_kv_splits=args.splits)
+        per96, _, _, _ = time_points([r96], stream, max(args.steps, 3), 2)
+        extra_pt = (98304, per96[0])
+        del r96
+
     # ---- max over ranks ----
     if world > 1:
         t = D.max_over_ranks([total_ms, e2e[1] if e2e else 0.0], dev)
@@ -571,24 +793,31 @@ def main():
                       "frac_of_sustained_peak": round(tf / sustained, 4)})
     cost_curve = None
     if len(prefixes) >= 3 and args.workload in ("cfg2", "cfg3", "cfg4"):
-        # the paper's linear latency model (its Eq. 2) and balance identity (its Eq. 3) on the measured curve
-        x = np.array(prefixes, dtype=np.float64); y = np.array(per_pt_ms, dtype=np.float64)
-        b, a = np.polyfit(x, y, 1)
-        r2 = 1.0 - float(((y - (a + b * x)) ** 2).sum() / max(((y - y.mean()) ** 2).sum(), 1e-30))
-        cost_curve = {"fit_ms": {"a": round(float(a), 5), "b_per_token": float(b), "r2": round(r2, 6)}}
-        steps_eq = np.diff(x)
-        if len(x) >= 3 and np.allclose(steps_eq, steps_eq[0]):
-            res = np.abs(y[:-2] + y[2:] - 2 * y[1:-1]) / (2 * y[1:-1])
-            cost_curve["eq3_residual_max"] = round(float(res.max()), 5)
+        cost_curve = fit_cost_curve(prefixes, per_pt_ms)
+        if extra_pt is not None:
+            # the paper's balance identity on evenly spaced points: the 96K point (timed outside the step) completes
+            # 0 / 32K / 64K / 96K / 128K
+            xs = sorted(set(prefixes) | {extra_pt[0]})
+            ys = [extra_pt[1] if x == extra_pt[0] else per_pt_ms[prefixes.index(x)] for x in xs]
+            even = fit_cost_curve(xs, ys)
+            cost_curve["eq3_residual_max"] = even.get("eq3_residual_max")
+            cost_curve["eq3_triples"] = even.get("eq3_triples")
+            cost_curve["eq3_points"] = "evenly spaced triples among %s (prefix %d timed outside the step: %.4f ms)" % (xs, extra_pt[0], extra_pt[1])
     # dominant kernel = the attention kernel at the longest prefix; its launch is timed together with the
     # ~10 us work-decomposition kernel that precedes it on the same stream
     i_top = int(np.argmax(flops_pt))
     ach = flops_pt[i_top] / (per_pt_ms[i_top] * 1e-3) / 1e12
-    # DRAM bytes of that launch from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum) of the same command
-    # restricted to the prefix: profiles/attn128_ws_cfg2.md; only known for the cfg2 / 131072 launch
-    traffic = 1708.1e6 if (args.workload == "cfg2" and prefixes[i_top] == 131072) else None
+    # DRAM bytes of that launch: from the record written beside the ncu summary of the same command (never a literal here)
+    traffic, traffic_source = None, None
+    if args.workload == "cfg2":
+        rec = read_traffic_record("attn128_ws_cfg2_traffic.txt")
+        if rec.get("prefix") == str(prefixes[i_top]) and args.splits == int(rec.get("num_kv_splits", "0")):
+            traffic = float(rec["dram_bytes_read"]) + float(rec["dram_bytes_write"])
+            traffic_source = "profiles/attn128_ws_cfg2_traffic.txt (ncu capture at commit %s)" % rec.get("commit", "?")
     roofline = {"bound": "tensor", "achieved": round(ach, 2), "peak": burst, "unit": "TFLOP/s",
-                "frac": round(ach / burst, 4), "traffic": traffic, "peak_source": "%s (burst bf16 matmul)" % peaks["_source"],
+                "frac": round(ach / burst, 4), "traffic": traffic, "traffic_source": traffic_source,
+                "algorithmic_bytes": int((prefixes[i_top] + chunk) * WL["hkv"] * 512 + chunk * WL["hq"] * (256 + 256 + 4))
+                if args.workload in ("cfg2", "cfg4") else None, "peak_source": "%s (burst bf16 matmul)" % peaks["_source"],
                 "frac_of_sustained": round(ach / sustained, 4), "kernel": "attention kernel, prefix %d" % prefixes[i_top]}
     line = {"metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True, "scaling": "weak",
@@ -606,6 +835,13 @@ def main():
         line["cpu_baseline"] = {"value": round(fl / dt / 1e12, 6), "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": "%d random (row, head) pairs of the chunk at prefix %d (%.1f s of CPU time)"
                                 % (n, int(prob_cpu.prefix_len[0]), dt)}
+    if args.workload == "cfg2" and world == 1 and not args.no_sweep and not args.prefixes:
+        del runners
+        if e2e:
+            del pipe, q_host, out_host, lse_host, k_host, v_host, k_pages, v_pages
+        base = None
+        torch.cuda.empty_cache()
+        line["configs"] = sweep_other_configs(dev, peaks, max(3, min(args.steps, 5)), max(3, args.warmup), not args.no_cpu_baseline)
     if world > 1:
         dist.destroy_process_group()
     print(json.dumps(line), flush=True)

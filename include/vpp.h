@@ -42,7 +42,8 @@ typedef enum {
     VPP_ERR_UNSUPPORTED = -2, /* head dims / block size this build has no kernel for   */
     VPP_ERR_WORKSPACE = -3,   /* workspace missing or smaller than the size query      */
     VPP_ERR_CUDA = -4,        /* a CUDA runtime / driver call failed                   */
-    VPP_ERR_TIMEOUT = -5      /* (device status only) a bounded device wait expired    */
+    VPP_ERR_TIMEOUT = -5      /* never returned by an entry point (none synchronises): the code a caller should
+                                 map a device status of VPP_DEV_TIMEOUT to once it has read *status          */
 } vpp_status;
 
 /* Values the device writes to *status (0 = success). */
@@ -73,10 +74,16 @@ typedef void *vpp_stream_t; /* a cudaStream_t */
  *              does not name are never read.
  * block_table  int32 [num_reqs, max_blocks_per_req]: physical block of logical block j of request r.
  *              NULL means contiguous: request r is "block" r and block_size is ignored (slot = token).
+ *              Then EVERY request's region must really hold max_seq_len slots (the kernels fetch whole
+ *              128-key tiles up to max_seq_len, so a loose bound would read past a shorter buffer):
+ *              k_block_stride >= max_seq_len * k_token_stride (the same for v), the last region
+ *              allocated in full.  With several requests the call checks the strides and returns
+ *              VPP_ERR_INVALID_ARG otherwise; the size of the allocation itself cannot be checked.
  * prefix_len   int32 [num_reqs], tokens of the request already cached before this chunk.
  * chunk_len    int32 [num_reqs], query rows of the request in this call (0 allowed).
  * total_q      host copy of sum(chunk_len); sizes out, lse and the workspace.
- * max_seq_len  host upper bound on prefix_len[r] + chunk_len[r].
+ * max_seq_len  host upper bound on prefix_len[r] + chunk_len[r]; for a contiguous cache also the
+ *              number of slots of each request's region (see block_table).
  * num_kv_splits  0: the library decides; 1: never split the key range; S > 1: split the key range of
  *              every query tile into up to S parts and merge them (split-KV).
  * out          bf16 [total_q, num_q_heads, head_dim_v], 16-byte aligned.
@@ -154,6 +161,27 @@ vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t n
                          float *lse, vpp_stream_t stream);
 
 /*
+ * Chunked-prefill attention over a RANGE of the cached keys, giving partial results -- the building block
+ * of a context-parallel prefix (the paper's background on context parallelism: the prefix KV cache is
+ * sharded along the sequence): each shard holder evaluates Eq. 1 over its own keys, the partials of all
+ * shards are gathered and vpp_lse_merge combines them.
+ *
+ * Same arguments as vpp_chunk_attn_fwd except that every query row only sees the keys at positions
+ * [kv_begin, kv_end) of its request (still subject to the causal rule), and that the results are written
+ * un-merged, in the layout vpp_lse_merge reads:
+ *   o_part    fp32 [total_q, num_q_heads, head_dim_v]: softmax-weighted values over the keys seen (normalised
+ *             within the range);  lse_part  fp32 [total_q, num_q_heads]: log-sum-exp over the keys seen.
+ * Stacking the o_part / lse_part of S ranges that tile [0, prefix_len + chunk_len) along a leading dimension
+ * gives vpp_lse_merge's o_parts / lse_parts, and its result equals vpp_chunk_attn_fwd's.
+ * args->out, args->lse and args->num_kv_splits are ignored; the workspace is still needed (size query with
+ * num_kv_splits = 1).  kv_begin must be a multiple of 128 and at most prefix_len[r] for every request with
+ * query rows (so that each row sees at least one key: otherwise VPP_DEV_BAD_LENGTHS, nothing written); kv_end
+ * must be a multiple of 128 or >= max_seq_len ("to the end").  Errors as vpp_chunk_attn_fwd.
+ */
+vpp_status vpp_chunk_attn_partial_fwd(const vpp_chunk_attn_args *args, int32_t kv_begin, int32_t kv_end,
+                                      float *o_part, float *lse_part, vpp_stream_t stream);
+
+/*
  * Same operation as vpp_chunk_attn_fwd, for callers that cannot obtain device memory themselves.
  * (The paper has no counterpart for this entry point: it is a packaging variant, not a method step.)
  *
@@ -168,7 +196,10 @@ vpp_status vpp_lse_merge(const float *o_parts, const float *lse_parts, int32_t n
  *  - Every device that loads the library holds the array (VPP_STATIC_SCRATCH_BYTES) until the
  *    process exits.
  *  - The first call on each device looks up the array's device address (a one-time set-up that is
- *    not a stream operation); make that first call before starting any stream capture.
+ *    not a stream operation); make that first call before starting any stream capture.  That look-up
+ *    may also be the moment the CUDA runtime loads this part of the library onto the device and
+ *    reserves the array, so make it at start-up, while device memory is still available: in a process
+ *    that has already handed out all device memory it can fail (VPP_ERR_CUDA, "out of memory").
  *  - With num_kv_splits = 0 the library's own split choice is dropped (the launch runs unsplit) when its partials do
  *    not fit the array.
  *  - A launch whose vpp_chunk_attn_workspace_size exceeds VPP_STATIC_SCRATCH_BYTES is refused
@@ -293,6 +324,27 @@ const char *vpp_last_error(void);
 
 /* Number of kernels the last successful vpp_chunk_attn_fwd on this host thread enqueued. */
 int32_t vpp_last_launch_count(void);
+
+/*
+ * The entry points describe q, the caches and their tiles to the copy engine with encoded tensor maps;
+ * encoded maps are kept in a process-wide cache keyed on (base address, extents, strides, tile), so a call
+ * that repeats an earlier call's buffers and shapes encodes nothing.  Process-wide totals so far (host
+ * pointers; either may be NULL): look-ups and driver encodes.
+ */
+void vpp_tensor_map_cache_stats(int64_t *lookups, int64_t *encodes);
+
+/*
+ * Test hooks (no attention arithmetic; not needed by a user of the library).
+ * vpp_test_tensor_map_cache: pure host code -- runs `repeats` identical look-ups plus two different ones
+ *   through the cache logic with a stand-in encoder; returns the number of encodes it took (3 when the
+ *   cache works) or a negative number on an inconsistency.
+ * vpp_test_bounded_wait: enqueues a one-CTA kernel that waits, with the bounded wait every kernel of this
+ *   library uses, at most limit_cycles (1 .. 2^31 SM clocks) for an arrival that never comes, then takes
+ *   the kernels' teardown: *status (device int32, zeroed by the caller) becomes VPP_DEV_TIMEOUT.  Nothing
+ *   is copied or multiplied, so nothing can fault or hang.
+ */
+int32_t vpp_test_tensor_map_cache(int32_t repeats);
+vpp_status vpp_test_bounded_wait(int32_t *status, int64_t limit_cycles, vpp_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -20,7 +20,9 @@ VPP_ERR_TIMEOUT = -5
 
 EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge", "vpp_status_string",
            "vpp_last_error", "vpp_last_launch_count", "vpp_chunk_attn_fwd_static", "vpp_static_scratch_bytes",
-           "vpp_static_last_error", "vpp_kv_append", "vpp_sparse_attn_workspace_size", "vpp_sparse_mla_fwd"]
+           "vpp_static_last_error", "vpp_kv_append", "vpp_sparse_attn_workspace_size", "vpp_sparse_mla_fwd",
+           "vpp_chunk_attn_partial_fwd", "vpp_tensor_map_cache_stats", "vpp_test_tensor_map_cache",
+           "vpp_test_bounded_wait"]
 
 
 class VppError(RuntimeError):
@@ -102,6 +104,15 @@ def load_library():
         lib.vpp_sparse_attn_workspace_size.argtypes = [ctypes.c_int32]
         lib.vpp_sparse_mla_fwd.restype = ctypes.c_int
         lib.vpp_sparse_mla_fwd.argtypes = [ctypes.POINTER(SparseAttnArgs), ctypes.c_void_p]
+        lib.vpp_chunk_attn_partial_fwd.restype = ctypes.c_int
+        lib.vpp_chunk_attn_partial_fwd.argtypes = [ctypes.POINTER(ChunkAttnArgs), ctypes.c_int32, ctypes.c_int32,
+                                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.vpp_tensor_map_cache_stats.restype = None
+        lib.vpp_tensor_map_cache_stats.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64)]
+        lib.vpp_test_tensor_map_cache.restype = ctypes.c_int32
+        lib.vpp_test_tensor_map_cache.argtypes = [ctypes.c_int32]
+        lib.vpp_test_bounded_wait.restype = ctypes.c_int
+        lib.vpp_test_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -173,6 +184,28 @@ def vpp_chunk_attn_fwd_static(args, stream=None):
     rc = lib.vpp_chunk_attn_fwd_static(ctypes.byref(args), ctypes.c_void_p(stream))
     if rc != VPP_OK:
         raise VppError(rc, "%s: %s" % (lib.vpp_status_string(rc).decode(), lib.vpp_static_last_error().decode()))
+
+
+def vpp_chunk_attn_partial_fwd(args, kv_begin, kv_end, o_part, lse_part, stream=None):
+    """Attention of the launch described by `args` over the cached keys [kv_begin, kv_end) only: writes the partial
+    results o_part fp32 [T, Hq, Dv] and lse_part fp32 [T, Hq] (one slice of vpp_lse_merge's inputs)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_chunk_attn_partial_fwd(ctypes.byref(args), int(kv_begin), int(kv_end), _ptr(o_part),
+                                                     _ptr(lse_part), ctypes.c_void_p(stream)))
+
+
+def vpp_tensor_map_cache_stats():
+    """(look-ups, driver encodes) of the library's tensor-map cache so far in this process."""
+    a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+    load_library().vpp_tensor_map_cache_stats(ctypes.byref(a), ctypes.byref(b))
+    return int(a.value), int(b.value)
+
+
+def vpp_test_bounded_wait(status, limit_cycles, stream=None):
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    _check(load_library().vpp_test_bounded_wait(_ptr(status), int(limit_cycles), ctypes.c_void_p(stream)))
 
 
 def vpp_static_scratch_bytes():

@@ -6,7 +6,6 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -20,6 +19,7 @@
 #include "kv_append.cuh"
 #include "merge.cuh"
 #include "prep.cuh"
+#include "wait_test.cuh"
 
 namespace {
 
@@ -84,23 +84,98 @@ EncodeFn get_encode() {
     return fn;
 }
 
+// Encoded tensor maps are cached: a serving loop calls with the same buffers and shapes again and again, and seven
+// to nine driver encodes per call are a visible part of a short launch.  A map depends only on (base address, rank,
+// extents, strides, box), so an entry never goes stale; the cache is a small direct-mapped table guarded by a mutex.
+struct TmapKey {
+    const void* base;
+    uint64_t dims[5];
+    uint64_t strides[4];
+    uint32_t box[5];
+    uint32_t rank;
+};
+using RawEncodeFn = bool (*)(CUtensorMap*, const TmapKey&);
+
+class TmapCache {
+public:
+    static constexpr int kSlots = 256;
+    bool get(const TmapKey& key, RawEncodeFn encode, CUtensorMap* out) {
+        const uint64_t h = hash(key);
+        Slot& sl = slots_[h % kSlots];
+        std::lock_guard<std::mutex> lk(mu_);
+        ++lookups_;
+        if (sl.valid && sl.hash == h && std::memcmp(&sl.key, &key, sizeof key) == 0) {
+            *out = sl.map;
+            return true;
+        }
+        CUtensorMap m;
+        if (!encode(&m, key)) return false;
+        ++encodes_;
+        sl.key = key;
+        sl.hash = h;
+        sl.map = m;
+        sl.valid = true;
+        *out = m;
+        return true;
+    }
+    void stats(int64_t* lookups, int64_t* encodes) {
+        std::lock_guard<std::mutex> lk(mu_);
+        *lookups = lookups_;
+        *encodes = encodes_;
+    }
+private:
+    struct Slot {
+        TmapKey key;
+        uint64_t hash = 0;
+        CUtensorMap map;
+        bool valid = false;
+    };
+    static uint64_t hash(const TmapKey& k) {   // FNV-1a over the key's bytes (the key is zero-initialised, padding included)
+        const unsigned char* b = reinterpret_cast<const unsigned char*>(&k);
+        uint64_t h = 1469598103934665603ull;
+        for (size_t i = 0; i < sizeof k; ++i) h = (h ^ b[i]) * 1099511628211ull;
+        return h;
+    }
+    std::mutex mu_;
+    Slot slots_[kSlots];
+    int64_t lookups_ = 0, encodes_ = 0;
+};
+TmapCache g_tmaps;
+
 // bf16 tensor, innermost dimension contiguous, 128-byte swizzle, zero fill out of bounds.
-bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-               const uint32_t* box) {
+bool encode_with_driver(CUtensorMap* m, const TmapKey& k) {
     EncodeFn enc = get_encode();
     if (!enc) return false;
     cuuint64_t gd[5], gs[4];
     cuuint32_t bx[5], es[5];
-    for (int i = 0; i < rank; ++i) {
-        gd[i] = dims[i];
-        bx[i] = box[i];
+    for (uint32_t i = 0; i < k.rank; ++i) {
+        gd[i] = k.dims[i];
+        bx[i] = k.box[i];
         es[i] = 1;
-        if (i > 0) gs[i - 1] = strides_bytes[i - 1];
+        if (i > 0) gs[i - 1] = k.strides[i - 1];
     }
-    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gd, gs, bx, es,
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, k.rank, const_cast<void*>(k.base), gd, gs, bx, es,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+
+TmapKey make_key(const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box) {
+    TmapKey k;
+    std::memset(&k, 0, sizeof k);
+    k.base = base;
+    k.rank = static_cast<uint32_t>(rank);
+    for (int i = 0; i < rank; ++i) {
+        k.dims[i] = dims[i];
+        k.box[i] = box[i];
+        if (i > 0) k.strides[i - 1] = strides_bytes[i - 1];
+    }
+    return k;
+}
+
+bool make_tmap(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+               const uint32_t* box) {
+    return g_tmaps.get(make_key(base, rank, dims, strides_bytes, box), encode_with_driver, m);
 }
 
 // ---- validation -------------------------------------------------------------------------------------
@@ -153,6 +228,11 @@ vpp_status validate_pointers(const vpp_chunk_attn_args* a) {
     for (int i = 0; i < 6; ++i)
         if (st[i] <= 0 || st[i] % 8 != 0)
             return fail(VPP_ERR_INVALID_ARG, "cache strides must be positive multiples of 8 elements");
+    if (a->block_table == nullptr && a->num_reqs > 1 &&
+        (a->k_block_stride < a->k_token_stride * a->max_seq_len || a->v_block_stride < a->v_token_stride * a->max_seq_len))
+        return fail(VPP_ERR_INVALID_ARG,
+                    "contiguous cache: every request's region must hold max_seq_len (%d) slots, but the block strides are "
+                    "shorter than max_seq_len token strides", a->max_seq_len);
     return VPP_OK;
 }
 
@@ -218,26 +298,12 @@ int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
 }
 
 // The pipelined kernel pairs two q-heads of one kv-head per work item; odd group sizes (MHA) take the
-// straight-line kernel, one head per item.  VPP_FORCE_SIMPLE=1 selects the straight-line kernel always
-// (a debugging aid; read once).
-bool force_simple() {
-    static const bool v = [] {
-        const char* e = std::getenv("VPP_FORCE_SIMPLE");
-        return e && e[0] == '1';
-    }();
-    return v;
-}
-bool use_ws_kernel(const vpp_chunk_attn_args* a) {
-    return !force_simple() && ((a->num_q_heads / a->num_kv_heads) % 2 == 0);
-}
+// straight-line kernel, one head per item.
+bool use_ws_kernel(const vpp_chunk_attn_args* a) { return (a->num_q_heads / a->num_kv_heads) % 2 == 0; }
 // The pair-of-SMs MLA kernel needs every 64-key group of a KV tile inside one page; smaller pages take the
-// single-CTA two-pass kernel.  VPP_MLA_SINGLE=1 forces the latter (debugging aid, read once).
+// single-CTA two-pass kernel.
 bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
-    static const bool force_single = [] {
-        const char* e = std::getenv("VPP_MLA_SINGLE");
-        return e && e[0] == '1';
-    }();
-    return !force_single && (a->block_table == nullptr || a->block_size >= 64) && sm_count_or_default() >= 2;
+    return (a->block_table == nullptr || a->block_size >= 64) && sm_count_or_default() >= 2;
 }
 int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     if (fam == Family::kMla576) return 1;
@@ -292,7 +358,39 @@ size_t vpp_chunk_attn_workspace_size(const vpp_chunk_attn_args* a) {
     return layout_for(a, fam).total;
 }
 
+namespace {
+// Key range of a partial launch, in KV tiles of kTileN keys (null: the whole causal range, final results).
+struct KeyRange {
+    int32_t begin_tile, end_tile;
+};
+vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, const KeyRange* range);
+}  // namespace
+
 vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_) {
+    return run_chunk_attn(a, stream_, nullptr);
+}
+
+vpp_status vpp_chunk_attn_partial_fwd(const vpp_chunk_attn_args* args, int32_t kv_begin, int32_t kv_end, float* o_part,
+                                      float* lse_part, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    if (!args) return fail(VPP_ERR_INVALID_ARG, "args is null");
+    if (kv_begin < 0 || kv_end <= kv_begin) return fail(VPP_ERR_INVALID_ARG, "need 0 <= kv_begin < kv_end");
+    if (kv_begin % vpp::kTileN != 0 || (kv_end % vpp::kTileN != 0 && kv_end < args->max_seq_len))
+        return fail(VPP_ERR_INVALID_ARG, "kv_begin must be a multiple of %d, and so must kv_end unless it is >= max_seq_len",
+                    vpp::kTileN);
+    if (args->total_q > 0 && (!o_part || !lse_part)) return fail(VPP_ERR_INVALID_ARG, "o_part and lse_part must be non-null");
+    vpp_chunk_attn_args b = *args;
+    b.num_kv_splits = 1;       // the caller's ranges are the split
+    b.out = o_part;            // (fp32 here; only checked for null and alignment)
+    b.lse = lse_part;
+    KeyRange r;
+    r.begin_tile = kv_begin / vpp::kTileN;
+    r.end_tile = static_cast<int32_t>((static_cast<int64_t>(kv_end) + vpp::kTileN - 1) / vpp::kTileN);
+    return run_chunk_attn(&b, stream_, &r);
+}
+
+namespace {
+vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, const KeyRange* range) {
     g_err[0] = 0;
     Family fam = Family::kNone;
     vpp_status st = validate(a, &fam);
@@ -432,6 +530,9 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     pp.max_units = L.max_units;
     pp.max_cost = (a->max_seq_len + vpp::kTileN - 1) / vpp::kTileN;
     if (pp.max_cost < 1) pp.max_cost = 1;
+    pp.partial = range ? 1 : 0;
+    pp.range_begin = range ? range->begin_tile : 0;
+    pp.range_end = range ? range->end_tile : 0;
     pp.header = reinterpret_cast<vpp::WorkHeader*>(ws + L.header);
     pp.units = reinterpret_cast<vpp::WorkUnit*>(ws + L.units);
     pp.row_splits = row_splits;
@@ -453,8 +554,9 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     ap.scale_log2e = a->softmax_scale * 1.4426950408889634f;
     ap.out = a->out;
     ap.lse = a->lse;
-    ap.o_parts = reinterpret_cast<float*>(ws + L.o_parts);
-    ap.lse_parts = reinterpret_cast<float*>(ws + L.lse_parts);
+    // a partial launch writes "split 0" of the caller's buffers, which have the merge kernel's input layout
+    ap.o_parts = range ? static_cast<float*>(a->out) : reinterpret_cast<float*>(ws + L.o_parts);
+    ap.lse_parts = range ? a->lse : reinterpret_cast<float*>(ws + L.lse_parts);
     ap.header_ro = pp.header;
     ap.header = pp.header;
     ap.units = pp.units;
@@ -522,6 +624,7 @@ vpp_status vpp_chunk_attn_fwd(const vpp_chunk_attn_args* a, vpp_stream_t stream_
     if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(ce));
     return VPP_OK;
 }
+}  // namespace
 
 vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t num_splits, int32_t total_q,
                          int32_t num_q_heads, int32_t head_dim_v, void* out, float* lse, vpp_stream_t stream_) {
@@ -709,11 +812,50 @@ vpp_status vpp_sparse_mla_fwd(const vpp_sparse_attn_args* a, vpp_stream_t stream
     return VPP_OK;
 }
 
-#ifdef VPP_TRACE
-// Timing experiment only: copies the clock stamps of CTA 0 to the host (synchronises).
-int vpp_debug_trace(long long* host_out, int n) {
-    return static_cast<int>(cudaMemcpyFromSymbol(host_out, vpp::g_trace, sizeof(long long) * n));
+
+void vpp_tensor_map_cache_stats(int64_t* lookups, int64_t* encodes) {
+    int64_t l = 0, e = 0;
+    g_tmaps.stats(&l, &e);
+    if (lookups) *lookups = l;
+    if (encodes) *encodes = e;
 }
-#endif
+
+int32_t vpp_test_tensor_map_cache(int32_t repeats) {
+    // the cache logic with a stand-in for the driver's encoder (pure host code)
+    static TmapCache cache;
+    auto fake = +[](CUtensorMap* m, const TmapKey& k) {
+        std::memset(m, 0, sizeof *m);
+        std::memcpy(m, &k, sizeof k < sizeof *m ? sizeof k : sizeof *m);
+        return true;
+    };
+    const uint64_t d1[3] = {128, 8, 1000}, s1[2] = {256, 2048}, d2[3] = {128, 8, 1001};
+    const uint32_t b1[3] = {64, 1, 128};
+    static const char anchor[64] = {0};
+    int64_t l0, e0, l1, e1;
+    cache.stats(&l0, &e0);
+    for (int i = 0; i < repeats; ++i) {
+        CUtensorMap m, ref;
+        const TmapKey k = make_key(anchor, 3, d1, s1, b1);
+        if (!cache.get(k, fake, &m)) return -1;
+        fake(&ref, k);
+        if (std::memcmp(&m, &ref, sizeof m) != 0) return -2;     // a hit must return what the encoder produced
+    }
+    CUtensorMap m;
+    if (!cache.get(make_key(anchor, 3, d2, s1, b1), fake, &m)) return -1;    // another extent: another map
+    if (!cache.get(make_key(anchor + 16, 3, d1, s1, b1), fake, &m)) return -1;   // another base: another map
+    cache.stats(&l1, &e1);
+    if (l1 - l0 != repeats + 2) return -3;
+    return static_cast<int32_t>(e1 - e0);
+}
+
+vpp_status vpp_test_bounded_wait(int32_t* status, int64_t limit_cycles, vpp_stream_t stream_) {
+    g_err[0] = 0;
+    if (!status || limit_cycles <= 0 || limit_cycles > (1ll << 31))
+        return fail(VPP_ERR_INVALID_ARG, "status must be non-null and limit_cycles in (0, 2^31]");
+    vpp::bounded_wait_test_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream_)>>>(status, limit_cycles);
+    const cudaError_t ce = cudaGetLastError();
+    if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "test kernel launch: %s", cudaGetErrorString(ce));
+    return VPP_OK;
+}
 
 }  // extern "C"

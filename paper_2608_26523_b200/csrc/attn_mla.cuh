@@ -196,10 +196,8 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             ok = mbar_wait(bar_k_empty + 8, (fill & 1) ^ 1, s_abort, 505);
                         }
                         for (int grp = 0; grp < 2 && ok; ++grp) {
-                            VPP_TR(3, j - t_lo, grp * 3 + 0);
                             ok = mbar_wait(bar_k_empty + 8 * grp, (fill & 1) ^ 1, s_abort, 503);
                             if (!ok) break;
-                            VPP_TR(3, j - t_lo, grp * 3 + 1);
                             const uint32_t full = bar_k_full + 8 * grp;
                             const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
                             mbar_arrive_expect_tx(full, (i1 - i0) * kMlaKSlab);
@@ -221,7 +219,6 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                                                     slot_in[q], 0, blk[q]);
                                 }
                             }
-                            VPP_TR(3, j - t_lo, grp * 3 + 2);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -303,7 +300,6 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const uint32_t tS = tmem_base + b * 64;
                     const bool has_next = jj + 1 < n;
                     bool early = false;
-                    VPP_TR(0, jj, 0);
                     if (has_next && mbar_try_wait(bar_k_full, (fill + 1) & 1)) {
                         // the non-value slabs of the next tile are already here: their score MMAs overlap the
                         // softmax of this tile (if they are not, P V of this tile must not wait for them)
@@ -317,17 +313,14 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         if (!ok) break;
                         ++vfix_it;
                     }
-                    VPP_TR(0, jj, 1);
                     ok = mbar_wait(bar_p_full + 8 * b, (tc >> 1) & 1, s_abort, 605);
                     if (!ok) break;
                     tc_fence_after();
-                    VPP_TR(0, jj, 2);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)
                         mma_ts_lh(tO, tS + kk * 8, v_lo + ((pass * 4 * kMlaKSlab + kk * 2048) >> 4), kHi, kIdescPV,
                                   (jj > 0 || kk > 0) ? 1u : 0u);
                     tc_commit(bar_k_empty + 8);
-                    VPP_TR(0, jj, 3);
                     ++fill;
                     ++tc;
                     if (has_next) {
@@ -336,13 +329,10 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                             if (!ok) break;
                             tc_commit(bar_k_empty);
                         }
-                        VPP_TR(0, jj, 4);
                         if (!mbar_wait(bar_k_full + 8, fill & 1, s_abort, 606)) { ok = false; break; }
-                        VPP_TR(0, jj, 5);
                         ok = issue_qk(tmem_base + (b ^ 1) * 64, pass, 1, fill);
                         if (!ok) break;
                         tc_commit(bar_s_full + 8 * (b ^ 1));
-                        VPP_TR(0, jj, 6);
                         if (jj + 2 == n && pass == 1) tc_commit(bar_q_empty);
                     } else {
                         tc_commit(bar_o_full);
@@ -382,7 +372,6 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!ok) break;
                     ++tc;
                     tc_fence_after();
-                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 0);
                     uint32_t s[64];
                     tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                     tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
@@ -421,7 +410,6 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         }
                     }
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 1);
                     float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
@@ -439,7 +427,6 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     l_run += sum0 + sum1;
                     tc_wait_st();
                     tc_fence_before();
-                    if (warp == 2 && lane == 0) VPP_TR(1, j - t_lo, 2);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_p_full + 8 * b);
                 }

@@ -437,7 +437,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 // S[b] was last read by the softmax of two tiles ago: its P is ready <=> that read is over
                 if (kc >= 2) ok = mbar_wait_cluster(bar_p_full + 8 * b, ((kc - 2) >> 1) & 1, s_abort, 820);
                 if (!ok) break;
-                VPP_TR(2, jj, 0);
                 ok = mbar_wait(bar_k_full, kpar, s_abort, 822);
                 if (!ok) break;
                 tc_fence_after();
@@ -493,7 +492,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                     ++vfix_it;
                 }
                 if (!ok) break;
-                VPP_TR(3, jj, 0);
                 ok = mbar_wait(bar_v_full, vpar, s_abort, 824);
                 if (!ok) break;
                 tc_fence_after();
@@ -504,7 +502,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 tc_fence_after();
                 if (jj == 0) pv_group_c(std::integral_constant<int, 1>{}, std::true_type{});
                 else pv_group_c(std::integral_constant<int, 1>{}, std::false_type{});
-                VPP_TR(0, jj, 5);
                 ++vc;
             }
         }
@@ -546,7 +543,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 ok = mbar_wait(bar_s_full + 8 * b, (tc >> 1) & 1, s_abort, 832);
                 if (!ok) break;
                 tc_fence_after();
-                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 0);
                 uint32_t s[64];
                 tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(s[0]));
                 tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(s[32]));
@@ -567,10 +563,8 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 const float mxa = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                                         fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
                 float mxb;
-                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 1);
                 ok = exchange(mxa, mxb);
                 if (!ok) break;
-                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 2);
                 const float m_new = fmaxf(fmaxf(mxa, mxb) * sc, m_ref);
                 const bool grow = (m_new - m_ref > 8.f) || (m_ref == -INFINITY && m_new != -INFINITY);
                 bool p_free = false;
@@ -609,7 +603,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                     pk[i >> 1] = pack_bf16x2(p0, p1);
                 }
                 l_run += sum0 + sum1;
-                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 3);
                 // P of the previous tile must have been consumed before its shared-memory rows are overwritten
                 if (tc > 0 && !p_free) {
                     ok = mbar_wait(bar_pv_done, (tc - 1) & 1, s_abort, 833);
@@ -622,7 +615,6 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
                 fence_proxy_async_smem();
                 tc_fence_before();
                 __syncwarp();
-                if (l128 == 0) VPP_TR(1, j - u.kv_begin, 4);
                 if (lane == 0) {
                     if (leader) mbar_arrive(bar_p_full + 8 * b);
                     else mbar_arrive_remote(bar_p_full + 8 * b, 0);

@@ -21,10 +21,7 @@ constexpr int kSimpleSmemBytes = 4 * 2 * kSlabBytes + 1024 /*align*/ + 256 /*bar
 // Which (unit, kv-head, q-head) a flat work index means.  Units arrive sorted by decreasing cost; inside
 // a block of kUnitBlock consecutive units the items are ordered kv-head-major so that CTAs running at
 // the same time read the same K/V pages (L2 reuse), while blocks keep the longest-first order.
-#ifndef VPP_UNIT_BLOCK
-#define VPP_UNIT_BLOCK 32
-#endif
-constexpr int kUnitBlock = VPP_UNIT_BLOCK;
+constexpr int kUnitBlock = 32;
 __device__ __forceinline__ void decode_item(int w, int num_units, int items_per_unit, int per_kv_head, int& unit,
                                             int& slot) {
     const int blk_items = kUnitBlock * items_per_unit;

@@ -32,23 +32,13 @@
 namespace vpp {
 
 constexpr int kWsThreads = 384;
-#ifndef VPP_WS_STAGES
-#define VPP_WS_STAGES 4
-#endif
-constexpr int kWsStages = VPP_WS_STAGES;      // 32 KB each
+constexpr int kWsStages = 4;                  // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 2048 /*barriers, ring, merge exchange*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
-#ifndef VPP_SPLIT_CHUNKS
-#define VPP_SPLIT_CHUNKS 1
-#endif
 // 0: P is handed to the MMA thread whole; c in 1..3: the first 32*c key columns are handed over early so that
 // O += P V can start on them while the rest of the exponentials are computed
-constexpr int kSplitChunks = VPP_SPLIT_CHUNKS;
-#ifndef VPP_EMU_EVERY
-#define VPP_EMU_EVERY 0
-#endif
-constexpr int kEmuEvery = VPP_EMU_EVERY;      // 0: all exponentials on the SFU (measured fastest so far)
+constexpr int kSplitChunks = 1;
 
 struct WsItem {
     WorkUnit u;
@@ -274,9 +264,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         const uint32_t dst = sKV + st * kTileBytes;
                         const uint32_t full = bar_kv_full + 8 * st;
                         if (lane == 0) {
-                            VPP_TR(3, j - u.kv_begin, which * 3 + 0);
                             ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
-                            VPP_TR(3, j - u.kv_begin, which * 3 + 1);
                             if (ok) {
                                 mbar_arrive_expect_tx(full, kTileBytes);
                                 const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
@@ -314,7 +302,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                     tma_load_4d(dst + o, tm, full, 0, slot_in, g, blk);
                                     tma_load_4d(dst + kSlabBytes + o, tm, full, 64, slot_in, g, blk);
                                 }
-                                VPP_TR(3, j - u.kv_begin, which * 3 + 2);
                             }
                         }
                         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -458,7 +445,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_kv_full + 8 * stV, (kv_it / kWsStages) & 1, 304);
                     if (!ok) break;
                     ++kv_it;
-                    if (lane == 0) VPP_TR(0, jj, 0);
                     if (tile0 + kTileN > u.kv_len) {
                         ok = wait1(bar_vfix + 24 * (vfix_it & 1), (vfix_it >> 1) & 1, 305);
                         if (!ok) break;
@@ -472,7 +458,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         if (!ok) break;
                         tc_fence_after();
                     }
-                    if (lane == 0) VPP_TR(0, jj, 1);
                     if (kSplitChunks > 0) {
                         ok = wait1(bar_p_part, p_it & 1, 311);
                         if (!ok) break;
@@ -485,26 +470,14 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else {
                         issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
                     }
-                    if (lane == 0) VPP_TR(0, jj, 2);
                     if (has_next) {
-#ifdef VPP_TRACE
-                        if (lane == 0) {
-                            VPP_TR(0, jj, 8);
-                            const bool first_try = mbar_try_wait(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1);
-                            VPP_TR(0, jj, 9);
-                            if (blockIdx.x == 0 && item_it == 1 && jj >= 8 && jj < 40) g_trace[(jj - 8) * 64 + 10] = first_try;
-                        }
-#endif
                         ok = wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 307);
                         if (!ok) break;
-                        if (lane == 0) VPP_TR(0, jj, 7);
                         tc_fence_after();
-                        if (lane == 0) VPP_TR(0, jj, 3);
                         if (lane == 0) {
                             issue_qk(tS0, q_lo0, sKV + stK * kTileBytes);
                             tc_commit(bar_s_full);
                         }
-                        if (lane == 0) VPP_TR(0, jj, 4);
                     } else if (lane == 0) {
                         tc_commit(bar_o_full);
                     }
@@ -518,7 +491,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ok = wait1(bar_p_full + 8, p_it1 & 1, 308);
                     if (!ok) break;
                     tc_fence_after();
-                    if (lane == 0) VPP_TR(0, jj, 5);
                     if (lane == 0) {
                         issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, kSplitChunks > 0 ? 2 * kSplitChunks : 0, 8);
                         tc_commit(bar_kv_empty + 8 * stV);
@@ -531,7 +503,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             tc_commit(bar_o_full + 8);
                         }
                     }
-                    if (lane == 0) VPP_TR(0, jj, 6);
                     if (has_next) ++kv_it;
                     ++p_it;
                     ++p_it1;
@@ -539,16 +510,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (!ok) break;
             }
         }
-#ifdef VPP_TRACE
-        else if (warp == 3 && lane == 0 && blockIdx.x == 0) {
-            // observer: when does each K/V stage of the first item really become full?
-            const uint32_t item_it = 1;
-            for (int i = 0; i < 2 * 40; ++i) {
-                if (!mbar_wait(bar_kv_full + 8 * (i % kWsStages), (i / kWsStages) & 1, s_abort, 999)) break;
-                VPP_TR(3, i >> 1, 6 + (i & 1));
-            }
-        }
-#endif
         // warps 2 and 3 have nothing to do until teardown
     } else {
         // ===================================== softmax groups =====================================
@@ -599,7 +560,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                     continue;
                 }
-                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 0);
                 uint32_t s[128];
                 const bool diag = tile0 + kTileN - 1 > u.pos0;  // keys beyond the row's position are masked
                 const int lim = my_pos - tile0;                 // columns <= lim are visible
@@ -610,7 +570,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 tc_wait_ld();
                 tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(s[64]));
                 tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(s[96]));
-                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 1);
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     if (hh == 1) tc_wait_ld();
@@ -651,7 +610,6 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
                 const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 2);
                 float sum0 = 0.f, sum1 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -660,9 +618,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     for (int i = 0; i < 32; i += 2) {
                         const float x0 = fmaf(__uint_as_float(s[c * 32 + i]), sc, -m_use);
                         const float x1 = fmaf(__uint_as_float(s[c * 32 + i + 1]), sc, -m_use);
-                        // optionally every kEmuEvery-th exponential runs on the FMA pipe instead of the SFU
-                        const float p0 = (kEmuEvery > 0 && (i % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x0) : ex2(x0);
-                        const float p1 = (kEmuEvery > 0 && ((i + 1) % kEmuEvery) == kEmuEvery - 1) ? ex2_poly(x1) : ex2(x1);
+                        const float p0 = ex2(x0), p1 = ex2(x1);
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
@@ -676,10 +632,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     }
                 }
                 l_run += sum0 + sum1;
-                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 3);
                 tc_wait_st();
                 tc_fence_before();
-                if ((warp & 3) == 0 && lane == 0) VPP_TR(1 + t, j - u.kv_begin, 4);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_p);
             }

@@ -59,20 +59,4 @@ struct AttnParams {
     int32_t* status;              // may be null
 };
 
-#ifdef VPP_TRACE
-// Timing experiment only (never part of the product build): clock64 stamps of CTA 0's roles.
-__device__ long long g_trace[64 * 32];
-#define VPP_TR(role, jj, k)                                                                     \
-    do {                                                                                        \
-        if (blockIdx.x == 0 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
-    } while (0)
-#define VPP_TR1(role, jj, k)                                                                    \
-    do {                                                                                        \
-        if (blockIdx.x == 1 && item_it == 1 && (jj) >= 8 && (jj) < 40) g_trace[((jj)-8) * 64 + (role)*16 + (k)] = clock64(); \
-    } while (0)
-#else
-#define VPP_TR(role, jj, k) do {} while (0)
-#define VPP_TR1(role, jj, k) do {} while (0)
-#endif
-
 }  // namespace vpp

@@ -55,8 +55,14 @@ vpp_status vpp_chunk_attn_fwd_static(const vpp_chunk_attn_args* args, vpp_stream
     vpp_chunk_attn_args a = *args;
     size_t need = vpp_chunk_attn_workspace_size(&a);
     if (need == 0) {
+        // invalid or unsupported arguments: report what the ordinary entry point reports for them (its argument checks
+        // come before the workspace check, so nothing is enqueued)
+        a.workspace = nullptr;
+        a.workspace_bytes = 0;
+        vpp_status st = vpp_chunk_attn_fwd(&a, stream);
+        if (st == VPP_OK || st == VPP_ERR_WORKSPACE) st = VPP_ERR_INVALID_ARG;
         snprintf(g_static_err, sizeof g_static_err, "invalid or unsupported arguments: %s", vpp_last_error());
-        return VPP_ERR_INVALID_ARG;
+        return st;
     }
     if (need > VPP_STATIC_SCRATCH_BYTES && a.num_kv_splits == 0) {
         // the split count was the library's choice (a throughput matter): an unsplit launch needs no partials

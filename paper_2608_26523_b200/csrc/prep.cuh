@@ -27,6 +27,9 @@ struct PrepParams {
     int32_t splits;      // S >= 1
     int32_t max_units;
     int32_t max_cost;    // ceil(max_seq_len / 128), >= 1
+    int32_t partial;     // 1: key-range restricted launch whose results are partial (o fp32, lse) of "split 0"
+    int32_t range_begin; // first KV tile of the key range (partial launches)
+    int32_t range_end;   // one past its last KV tile
     WorkHeader* header;
     WorkUnit* units;
     int32_t* row_splits;  // [total_q], only written when splits > 1
@@ -106,7 +109,9 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
         if (r < p.num_reqs) {
             const int P = p.prefix_len[r];
             c = p.chunk_len[r];
-            if (P < 0 || c < 0 || static_cast<long long>(P) + c > p.max_seq_len) {
+            // (a key range must start inside every request's prefix, so that each query row sees at least one of its keys)
+            if (P < 0 || c < 0 || static_cast<long long>(P) + c > p.max_seq_len ||
+                (p.partial && c > 0 && P < p.range_begin * kTileN)) {
                 atomicExch(&s_error, 1 /* VPP_DEV_BAD_LENGTHS */);
                 c = 0;
             }
@@ -178,10 +183,15 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
             const int rows = (C - row_off) < kTileM ? (C - row_off) : kTileM;
             const int pos0 = P + row_off;
             const int n_tiles = (pos0 + rows + kTileN - 1) / kTileN;
-            const int nsplit = tile_num_splits(pos0, p.splits);
+            const int nsplit = p.partial ? 1 : tile_num_splits(pos0, p.splits);
             for (int s = 0; s < nsplit; ++s) {
                 int kb, ke;
-                split_range(pos0, n_tiles, nsplit, s, kb, ke);
+                if (p.partial) {
+                    kb = p.range_begin;
+                    ke = n_tiles < p.range_end ? n_tiles : p.range_end;
+                } else {
+                    split_range(pos0, n_tiles, nsplit, s, kb, ke);
+                }
                 // single-token units go to the end of the list (each part ordered by decreasing cost): the attention
                 // kernels may run them with the q-heads of a kv-head packed into one tile
                 const int bin = cost_bin(ke - kb, p.max_cost) + (rows == 1 ? kCostBins : 0);
@@ -197,7 +207,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
                         u.pos0 = pos0;
                         u.kv_begin = kb;
                         u.kv_end = ke;
-                        u.split = (nsplit > 1) ? s : -1;
+                        u.split = (nsplit > 1 || p.partial) ? s : -1;
                         u.kv_len = P + C;
                         p.units[slot] = u;
                     }

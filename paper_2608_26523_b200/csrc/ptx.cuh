@@ -53,7 +53,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // and returns false; the caller then drains and leaves through the normal teardown.
 constexpr long long kWaitLimitCycles = 1ll << 31;  // about a second at B200 clocks
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where) {
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where,
+                                              long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     int spins = 0;
@@ -61,12 +62,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63) == 0) {
             if (*abort_flag != 0) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 atomicCAS(const_cast<int*>(abort_flag), 0, where);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int where) {
+    return mbar_wait_for(bar, parity, abort_flag, where, kWaitLimitCycles);
 }
 
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA / tcgen05.mma operands)
@@ -103,14 +107,6 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* m, 
         "[%2];" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
-}
-
-// L2 prefetch of a rank-5 box (no shared-memory destination, no barrier)
-__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* m, int c0, int c1, int c2, int c3, int c4) {
-    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global [%0, {%1, %2, %3, %4, %5}];" ::"l"(
-                     reinterpret_cast<uint64_t>(m)),
-                 "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-                 : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -258,20 +254,6 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-// 2^x on the FMA pipe (for x <= ~100): floor/fraction split with a round-down magic add, degree-4
-// minimax polynomial for 2^f on [0,1) (max relative error 2.7e-6, mean 4e-8), exponent patched in with
-// an integer add.  Used for a fraction of the softmax exponentials to take load off the SFU (16
-// ex2/clk/SM), which otherwise limits the softmax at head_dim 128.
-__device__ __forceinline__ float ex2_poly(float x) {
-    x = fmaxf(x, -126.f);
-    const float xf = __fadd_rd(x, 12582912.f);  // 1.5 * 2^23: the low mantissa bits now hold floor(x)
-    const float f = x - (xf - 12582912.f);
-    float p = fmaf(0.013534167781472206f, f, 0.05201146379113197f);
-    p = fmaf(p, f, 0.2414427548646927f);
-    p = fmaf(p, f, 0.6930038332939148f);
-    p = fmaf(p, f, 1.0000026226043701f);
-    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xf) << 23));
 }
 // Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization attribute may start
 // while its predecessor in the stream still runs; pdl_wait() returns once that predecessor has completed and its

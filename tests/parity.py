@@ -86,3 +86,36 @@ def sample_rows(prob_cpu, n_random=256, seed=0):
         for _ in range(max(1, n_random // max(prob_cpu.num_reqs, 1))):
             trip.append((r, int(rng.integers(0, C)), int(rng.integers(0, hq))))
     return np.array(sorted(set(trip)), dtype=np.int32)
+
+
+def tile_rows(prob_cpu, per="pair", seed=0, every=1):
+    """One random (row, head) per work item of the launch: for every 128-row query tile of every request, one row
+    of the tile and one head out of each head group -- "pair": each pair of q-heads (the items of the d = 128
+    kernel); "kvhead": each kv-head's group; "tile": one head of all.  `every` > 1 keeps every n-th tile only."""
+    rng = np.random.default_rng(seed)
+    hq, hkv = prob_cpu.num_q_heads, prob_cpu.num_kv_heads
+    groups = {"pair": [(h, min(h + 2, hq)) for h in range(0, hq, 2)],
+              "kvhead": [(g * (hq // hkv), (g + 1) * (hq // hkv)) for g in range(hkv)],
+              "tile": [(0, hq)]}[per]
+    trip = []
+    for r in range(prob_cpu.num_reqs):
+        C = int(prob_cpu.chunk_len[r])
+        for k, t0 in enumerate(range(0, C, 128)):
+            if k % every:
+                continue
+            for lo, hi in groups:
+                trip.append((r, int(rng.integers(t0, min(t0 + 128, C))), int(rng.integers(lo, hi))))
+    return np.array(sorted(set(trip)), dtype=np.int32).reshape(-1, 3)
+
+
+def all_heads_of_rows(prob_cpu, n_rows=8, seed=0):
+    """Every q-head of n_rows random rows per request (first and last row included)."""
+    rng = np.random.default_rng(seed)
+    trip = []
+    for r in range(prob_cpu.num_reqs):
+        C = int(prob_cpu.chunk_len[r])
+        if C == 0:
+            continue
+        rows = {0, C - 1} | {int(x) for x in rng.integers(0, C, max(n_rows - 2, 0))}
+        trip += [(r, i, h) for i in sorted(rows) for h in range(prob_cpu.num_q_heads)]
+    return np.array(sorted(set(trip)), dtype=np.int32).reshape(-1, 3)

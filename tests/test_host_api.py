@@ -206,3 +206,65 @@ def test_split_choice_fills_whole_waves(lib):
     assert _chosen_splits(64, 64, 64, 4, 32769) == 4       # 256 items
     assert _chosen_splits(256, 256, 64, 8, 8193) == 1      # 2048 items
     assert _chosen_splits(32, 32, 64, 8, 8193) == 1        # 256 short items: the start-up of more units outweighs the wave
+
+
+def test_tensor_map_cache_encodes_once_per_distinct_map(lib):
+    """The cache logic with a stand-in for the driver's encoder: five identical look-ups, one with another extent and
+    one with another base address take three encodes, and a hit returns the bytes the encoder produced."""
+    assert lib.vpp_test_tensor_map_cache(5) == 3
+    assert lib.vpp_test_tensor_map_cache(7) == 0          # everything is cached by now
+    lookups, encodes = api.vpp_tensor_map_cache_stats()   # the library's own cache: untouched without a launch
+    assert lookups >= 0 and encodes <= lookups
+
+
+def test_contiguous_cache_regions_must_hold_max_seq_len_slots(lib):
+    """Two requests in an unpaged cache whose regions are 40 slots apart, with max_seq_len = 64: the kernels would fetch
+    key tiles up to slot 64 of the last region, past the allocation.  The call refuses on the host; nothing is launched."""
+    p = W.make_problem(8, [10, 12], [20, 8], 4, 2, 128, 128, block_size=None)
+    slots = p.k_cache.shape[1]
+    a = api.make_args(p.q, p.k_cache, p.v_cache, None, p.prefix_len, p.chunk_len, 0, slots + 24, p.scale)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8)
+    out = torch.zeros(28, 4, 128, dtype=torch.bfloat16)
+    a.workspace, a.workspace_bytes, a.out = ws.data_ptr() + (-ws.data_ptr() % 256), 1 << 19, out.data_ptr()
+    with pytest.raises(api.VppError) as ei:
+        api.vpp_chunk_attn_fwd(a, stream=0)
+    assert ei.value.status == api.VPP_ERR_INVALID_ARG and "max_seq_len" in str(ei.value)
+
+
+def test_unsupported_head_dim_gives_the_same_status_from_both_entry_points(lib):
+    a = small_args(dqk=96, dv=96)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8)
+    out = torch.zeros(20, 4, 96, dtype=torch.bfloat16)
+    a.workspace, a.workspace_bytes, a.out = ws.data_ptr() + (-ws.data_ptr() % 256), 1 << 19, out.data_ptr()
+    assert api.vpp_chunk_attn_workspace_size(a) == 0
+    for call in (api.vpp_chunk_attn_fwd, api.vpp_chunk_attn_fwd_static):
+        with pytest.raises(api.VppError) as ei:
+            call(a, stream=0)
+        assert ei.value.status == api.VPP_ERR_UNSUPPORTED, call.__name__
+    b = small_args()
+    b.num_kv_heads = 3                                  # 4 q-heads over 3 kv-heads: invalid, not unsupported
+    for call in (api.vpp_chunk_attn_fwd, api.vpp_chunk_attn_fwd_static):
+        with pytest.raises(api.VppError) as ei:
+            call(b, stream=0)
+        assert ei.value.status == api.VPP_ERR_INVALID_ARG, call.__name__
+
+
+@pytest.mark.parametrize("kv_begin,kv_end", [(-128, 128), (64, 256), (128, 128), (256, 128), (0, 200)])
+def test_partial_entry_point_checks_its_key_range(lib, kv_begin, kv_end):
+    p = W.make_problem(9, [600], [100], 4, 2, 128, 128, block_size=64)
+    a = api.make_args(p.q, p.k_cache, p.v_cache, p.block_table, p.prefix_len, p.chunk_len, p.block_size,
+                      p.max_seq_len, p.scale)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8)
+    a.workspace, a.workspace_bytes = ws.data_ptr() + (-ws.data_ptr() % 256), 1 << 19
+    o = torch.zeros(100, 4, 128, dtype=torch.float32)
+    l = torch.zeros(100, 4, dtype=torch.float32)
+    with pytest.raises(api.VppError) as ei:
+        api.vpp_chunk_attn_partial_fwd(a, kv_begin, kv_end, o, l, stream=0)
+    assert ei.value.status == api.VPP_ERR_INVALID_ARG
+
+
+def test_bounded_wait_hook_checks_its_arguments(lib):
+    assert lib.vpp_test_bounded_wait(None, 1000, None) == api.VPP_ERR_INVALID_ARG
+    st = torch.zeros(1, dtype=torch.int32)
+    assert lib.vpp_test_bounded_wait(st.data_ptr(), 0, None) == api.VPP_ERR_INVALID_ARG
+    assert lib.vpp_test_bounded_wait(st.data_ptr(), 1 << 40, None) == api.VPP_ERR_INVALID_ARG

@@ -5,12 +5,15 @@ running inside a framework's memory-planned region, or a server that gave all de
 start-up: they pass inputs and outputs, and the library's built-in scratch array replaces the
 workspace.  The test calls it through the C ABI twice in a row on a launch that really uses scratch
 (forced split-KV: work list, per-row split counts and fp32 partials) and compares both results with the
-ordinary entry point's, then checks that an oversized launch is refused cleanly.
+ordinary entry point's and with the CPU oracle (every element), checks that further calls leave the device's free memory
+and torch's allocator untouched, then that an oversized launch is refused cleanly.
 """
 import pytest
 import torch
 
+import oracle
 from paper_2608_26523_b200 import api, workloads as W
+from parity import compare
 
 pytestmark = pytest.mark.gpu
 
@@ -31,11 +34,15 @@ def _launch(prob, static, num_kv_splits):
 
 
 def test_static_scratch_matches_workspace_entry_point_twice():
-    prob = W.make_problem(9001, [900, 0, 260], [300, 140, 77], 8, 2, 128, 128, block_size=64).to("cuda")
+    prob_cpu = W.make_problem(9001, [900, 0, 260], [300, 140, 77], 8, 2, 128, 128, block_size=64)
+    prob = prob_cpu.to("cuda")
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
     ref_out, ref_lse = _launch(prob, static=False, num_kv_splits=3)
     assert torch.isfinite(ref_out).all()
     for call in range(2):                                    # the second call finds the first one's leftovers
         out, lse = _launch(prob, static=True, num_kv_splits=3)
+        # against the definition: every element, with the tolerances of the parity suite
+        compare(out, lse, prob_cpu, rows, "static entry point, call %d" % call)
         # same kernels, same work list: the results agree to the tolerance of the parity tests (they are in
         # fact identical up to the order in which equal-cost work units were listed)
         assert (out - ref_out).abs().max().item() <= 1e-2, "call %d" % call
@@ -45,6 +52,26 @@ def test_static_scratch_matches_workspace_entry_point_twice():
     _launch(other, static=True, num_kv_splits=0)
     out, lse = _launch(prob, static=True, num_kv_splits=3)
     assert (out - ref_out).abs().max().item() <= 1e-2
+
+
+def test_static_entry_point_allocates_nothing_after_its_first_call():
+    """The first call on a device resolves the scratch array's address (and may make the runtime load that part of the
+    library); from then on a call that really uses the scratch (split-KV partials) must leave the device's free memory
+    and torch's allocator exactly as they were."""
+    prob = W.make_problem(9005, [700], [400], 8, 2, 128, 128, block_size=64).to("cuda")
+    runner = api.ChunkAttn(prob, num_kv_splits=4)
+    runner.args.workspace, runner.args.workspace_bytes = None, 0
+    api.vpp_chunk_attn_fwd_static(runner.args)               # first call: set-up included
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        api.vpp_chunk_attn_fwd_static(runner.args)
+    torch.cuda.synchronize()
+    assert int(runner.status.item()) == 0
+    free1, _ = torch.cuda.mem_get_info()
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert free1 == free0, "device free memory changed by %d bytes across static calls" % (free0 - free1)
 
 
 def test_static_scratch_refuses_oversized_launch():
