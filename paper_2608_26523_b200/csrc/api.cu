@@ -310,6 +310,25 @@ int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     return use_ws_kernel(a) ? 2 : 1;
 }
 
+using MergeKernel = void (*)(const float*, const float*, int, long long, int, int, const int32_t*, __nv_bfloat16*, float*);
+// The kernel and the grid for a merge of `splits` partials of total_q x num_q_heads rows of head_dim_v features.
+MergeKernel pick_merge_kernel(int splits, long long total_q, int num_q_heads, int head_dim_v, int sms, unsigned* blocks) {
+    const long long pairs = total_q * num_q_heads;
+    const long long pieces = pairs * (head_dim_v / 4);
+    if (splits <= vpp::kMergeSmallMax && head_dim_v % 4 == 0 && pieces < (1ll << 31)) {
+        long long b = (pieces + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+        if (b > 12ll * sms) b = 12ll * sms;
+        *blocks = static_cast<unsigned>(b);
+        if (splits <= 2) return vpp::lse_merge_small_kernel<2, 4>;
+        if (splits <= 4) return vpp::lse_merge_small_kernel<4, 2>;
+        return vpp::lse_merge_small_kernel<8, 1>;
+    }
+    long long b = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
+    if (b > 8ll * sms) b = 8ll * sms;
+    *blocks = static_cast<unsigned>(b);
+    return vpp::lse_merge_kernel<2, 4>;
+}
+
 vpp::WorkspaceLayout layout_for(const vpp_chunk_attn_args* a, Family fam) {
     vpp::WorkspaceLayout L{};
     const int S = choose_splits(a, heads_per_item(a, fam));
@@ -600,19 +619,18 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
 
     // ---- merge of split partials ----
     if (L.splits > 1) {
-        const long long pairs = static_cast<long long>(a->total_q) * a->num_q_heads;
-        long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
-        if (blocks > 8ll * sms) blocks = 8ll * sms;
+        unsigned blocks = 1;
+        const MergeKernel mk = pick_merge_kernel(L.splits, a->total_q, a->num_q_heads, a->head_dim_v, sms, &blocks);
         cudaLaunchAttribute attr{};
         attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr.val.programmaticStreamSerializationAllowed = 1;
         cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+        cfg.gridDim = dim3(blocks);
         cfg.blockDim = dim3(vpp::kMergeThreads);
         cfg.stream = stream;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        ce = cudaLaunchKernelEx(&cfg, vpp::lse_merge_kernel, static_cast<const float*>(ap.o_parts),
+        ce = cudaLaunchKernelEx(&cfg, mk, static_cast<const float*>(ap.o_parts),
                                 static_cast<const float*>(ap.lse_parts), static_cast<int>(L.splits),
                                 static_cast<long long>(a->total_q), static_cast<int>(a->num_q_heads),
                                 static_cast<int>(a->head_dim_v), static_cast<const int32_t*>(row_splits),
@@ -638,13 +656,10 @@ vpp_status vpp_lse_merge(const float* o_parts, const float* lse_parts, int32_t n
     if ((reinterpret_cast<uintptr_t>(o_parts) | reinterpret_cast<uintptr_t>(out)) & 15u)
         return fail(VPP_ERR_INVALID_ARG, "o_parts and out must be 16-byte aligned");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const long long pairs = static_cast<long long>(total_q) * num_q_heads;
-    long long blocks = (pairs * 32 + vpp::kMergeThreads - 1) / vpp::kMergeThreads;
-    const long long cap = 8ll * sm_count_or_default();
-    if (blocks > cap) blocks = cap;
-    vpp::lse_merge_kernel<<<static_cast<unsigned>(blocks), vpp::kMergeThreads, 0, stream>>>(
-        o_parts, lse_parts, num_splits, total_q, num_q_heads, head_dim_v, nullptr, static_cast<__nv_bfloat16*>(out),
-        lse);
+    unsigned blocks = 1;
+    const MergeKernel mk = pick_merge_kernel(num_splits, total_q, num_q_heads, head_dim_v, sm_count_or_default(), &blocks);
+    mk<<<blocks, vpp::kMergeThreads, 0, stream>>>(o_parts, lse_parts, num_splits, total_q, num_q_heads, head_dim_v, nullptr,
+                                                  static_cast<__nv_bfloat16*>(out), lse);
     cudaError_t ce = cudaGetLastError();
     if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "merge launch: %s", cudaGetErrorString(ce));
     return VPP_OK;
