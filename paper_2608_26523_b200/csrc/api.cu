@@ -502,12 +502,13 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
                                 static_cast<uint64_t>(a->num_q_heads)};
         const uint64_t sq[3] = {static_cast<uint64_t>(a->head_dim_qk) * a->num_q_heads * 2, 128,
                                 static_cast<uint64_t>(a->head_dim_qk) * 2};
-        const uint32_t bq[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // all nine slabs in one copy
+        const uint32_t bq[4] = {vpp::kMla2BoxCols, vpp::kMla2BoxRows, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // all nine slabs in one copy
         const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
                                static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
         const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
                                 static_cast<uint64_t>(a->k_block_stride) * 2};
-        const uint32_t b3[5] = {64, 64, 3, 1, 1}, b2[5] = {64, 64, 2, 1, 1};
+        const uint32_t b3[5] = {vpp::kMla2BoxCols, vpp::kMla2BoxRows, vpp::kKG, 1, 1};               // one K hand-back group
+        const uint32_t b2[5] = {vpp::kMla2BoxCols, vpp::kMla2BoxRows, vpp::kMla2VBoxSlabs, 1, 1};    // one V chunk
         if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) ||
             !make_tmap(&tm_k93, a->k_cache, 5, d, sk, b3) || !make_tmap(&tm_k92, a->k_cache, 5, d, sk, b2))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");

@@ -50,6 +50,41 @@ constexpr int kVG = 2;  // V chunks per hand-back group (2 groups per tile: key 
 constexpr int kKGroups = kMlaSlabs / kKG, kVGroups = kMla2VChunks / kVG;
 constexpr int kMla2SmemBytes = kMla2QBytes + kMla2KBytes + kMla2VBytes + kMla2PBytes + 1024 /*align*/ + 1536;
 
+// ---- the pair protocol as checkable facts --------------------------------------------------------------------
+// Copy boxes (elements of the tensor maps the host encodes; the host uses these constants):
+constexpr int kMla2BoxCols = 64, kMla2BoxRows = 64;                       // 64 features x 64 rows / keys per slab
+constexpr int kMla2QBoxBytes = kMla2BoxCols * kMla2BoxRows * kMlaSlabs * 2;   // one copy: all nine slabs of a CTA's 64 rows
+constexpr int kMla2KBoxBytes = kMla2BoxCols * kMla2BoxRows * kKG * 2;         // one copy: one K hand-back group of a CTA
+constexpr int kMla2VBoxSlabs = 2;                                             // one copy: one V chunk = 2 slabs x 64 keys
+constexpr int kMla2VBoxBytes = kMla2BoxCols * kMla2BoxRows * kMla2VBoxSlabs * 2;
+// Bytes announced on a barrier = sum of the boxes of the copies that post on it:
+//   bar_q_full            2 CTAs x 1 copy  of kMla2QBoxBytes         (announced: 2 * kMla2QBytes)
+//   bar_k_full[g]         2 CTAs x 1 copy  of kMla2KBoxBytes         (announced: 2 * kKG * 8192)
+//   bar_v_full[g]         2 CTAs x kVG copies of kMla2VBoxBytes      (announced: 2 * kVG * kMla2VChunk);
+//                         on a tile past the end of the sequence each CTA lands its own kVG copies on a barrier of its
+//                         own (announced there: kVG * kMla2VChunk)
+static_assert(kMla2QBoxBytes == kMla2QBytes, "Q: one copy per CTA fills the CTA's Q buffer");
+static_assert(kMla2KBoxBytes == kKG * 8192, "K: a group's copy is what the producer announces per CTA");
+static_assert(kMla2VBoxBytes == kMla2VChunk, "V: a chunk's copy is what the producer announces per chunk");
+static_assert(kKG * kKGroups == kMlaSlabs && kVG * kVGroups == kMla2VChunks, "groups tile the K slabs / V chunks");
+static_assert(2 * kMla2QBytes < (1 << 20) && 2 * kKG * 8192 < (1 << 20) && 2 * kVG * kMla2VChunk < (1 << 20),
+              "a barrier's pending byte count must stay below 2^20");
+// Arrivals per phase: bar_p_full = one per softmax warp of both CTAs (4 + 4); bar_xchg = every softmax thread of a CTA;
+// bar_vfix = one per CTA; every other barrier has a single arrival (a producer's announce or a tcgen05.commit).
+constexpr int kMla2SoftmaxWarps = 4;
+constexpr int kMla2PFullArrivals = 2 * kMla2SoftmaxWarps, kMla2XchgArrivals = 32 * kMla2SoftmaxWarps;
+// Which commit hands back what (all commits are multicast to both CTAs, issued by the leader's two MMA threads; a
+// commit covers only the MMAs of the thread that issues it):
+//   score thread, after K group g < last:  bar_k_empty[g]   -> K group g may be refilled
+//   score thread, after the last K group:  bar_s_full[b]    -> scores of S[b] ready; last K group free; Q free after an item
+//   P V thread,   after V group g < last:  bar_v_empty[g]   -> V group g may be refilled
+//   P V thread,   after the last V group:  bar_pv_done      -> last V group free; P free; O quiescent / complete
+// Tensor-memory columns of a CTA (512 allocated): S[0] 0..63, S[1] 64..127, O columns 128..255 and 256..383.
+constexpr int kMla2TmemS = 0, kMla2TmemO0 = 128, kMla2TmemO1 = 256, kMla2TmemEnd = 384;
+static_assert(kMla2TmemS + 2 * 64 <= kMla2TmemO0 && kMla2TmemO0 + 128 <= kMla2TmemO1 && kMla2TmemO1 + 128 <= kMla2TmemEnd &&
+              kMla2TmemEnd <= 512, "tensor-memory regions do not overlap");
+static_assert(kMla2SmemBytes <= 232448, "shared memory of one CTA");
+
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -197,10 +232,10 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         mbar_init(bar_pv_done, 1);
         mbar_init(bar_s_full, 1);
         mbar_init(bar_s_full + 8, 1);
-        mbar_init(bar_p_full, 8);
-        mbar_init(bar_p_full + 8, 8);
+        mbar_init(bar_p_full, kMla2PFullArrivals);
+        mbar_init(bar_p_full + 8, kMla2PFullArrivals);
         mbar_init(bar_vfix, 2);     // one arrival per CTA
-        mbar_init(bar_xchg, 128);
+        mbar_init(bar_xchg, kMla2XchgArrivals);
         for (int i = 0; i < kKGroups; ++i) {
             mbar_init(bar_k_full + 8 * i, 1);
             mbar_init(bar_k_empty + 8 * i, 1);
@@ -458,7 +493,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         constexpr uint32_t kHi = desc_hi_sw128(1024);
         const uint32_t p_lo = desc_lo_sw128(sP, 16);
         const uint32_t v_lo = desc_lo_sw128(sV, 8192);  // MN-major: 64-column groups 8 KB apart
-        const uint32_t tO0 = tmem_base + 128, tO1 = tmem_base + 256;
+        const uint32_t tO0 = tmem_base + kMla2TmemO0, tO1 = tmem_base + kMla2TmemO1;
         uint32_t vc = 0, vfix_it = 0, item_it = 0;   // vc: P V tiles issued so far (all items)
         bool ok = true;
         // O += P V for V group g: chunk c = (key half c >> 1, output half c & 1)
@@ -511,7 +546,7 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
         const int row = l128 & 63;                     // row of this CTA's 64
         const int half = l128 >> 6;                    // which 64 key columns of the tile
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-        const uint32_t tO0 = tmem_base + 128 + lane_off, tO1 = tmem_base + 256 + lane_off;
+        const uint32_t tO0 = tmem_base + kMla2TmemO0 + lane_off, tO1 = tmem_base + kMla2TmemO1 + lane_off;
         uint8_t* p_row = gen_base + kMla2QBytes + kMla2KBytes + kMla2VBytes + half * 8192 + row * 128;
         uint32_t tc = 0, x_it = 0, item_it = 0;
         const float sc = p.scale_log2e;
