@@ -288,6 +288,46 @@ def sweep_other_configs(dev, peaks, steps, warmup, with_cpu):
     return out
 
 
+def bench_groups(args):
+    """Group sizes: the same chunk (8192 rows at prefix 32768, d = 128, 128-token pages) with MHA, an odd group and an even
+    group -- work items are two q-heads of a kv-head over 128 rows (even groups) or two 128-row tiles of one q-head (odd
+    groups, MHA included); both run the pipelined kernel."""
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    prefix, chunk = (int(args.prefixes.split(",")[0]) if args.prefixes else 32768), 8192
+    cases = [("MHA: Hq=32 Hkv=32", 32, 32), ("odd group: Hq=24 Hkv=8 (G=3)", 24, 8), ("even group: Hq=32 Hkv=8 (G=4)", 32, 8),
+             ("MQA-like: Hq=32 Hkv=1 (G=32)", 32, 1)]
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches = 0
+    for desc, hq, hkv in cases:
+        prob = W.make_problem(W.BASE_SEED + 500 + hkv, [prefix], [chunk], hq, hkv, 128, 128, block_size=128, device=dev)
+        runner = api.ChunkAttn(prob, num_kv_splits=args.splits)
+        per, step_ms, nl, _ = time_points([runner], stream, max(args.steps, 5), max(args.warmup, 3))
+        launches += nl * max(args.steps, 5)
+        tf = prob.flops() / (per[0] * 1e-3) / 1e12
+        rows.append({"case": desc, "ms": round(per[0], 4), "tflops": round(tf, 1), "frac_of_burst": round(tf / peaks["bf16_tflops"], 4)})
+        del prob, runner
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[0]
+    print(json.dumps({"metric": "chunk attention TFLOP/s by group size (1 B200)", "value": top["tflops"], "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": top["ms"], "higher_is_better": True, "dtype": "bf16",
+                      "data": "synthetic", "vs_baseline": None,
+                      "config": {"workload": "groups; chunk %d at prefix %d, d=128, 128-token pages; %s" % (chunk, prefix, top["case"]),
+                                 "l2": "K/V of the MHA case (%d MB) exceeds the L2" % ((prefix + chunk) * 32 * 512 // 1000000)},
+                      "cases": rows,
+                      "roofline": {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": UNIT,
+                                   "frac": top["frac_of_burst"], "traffic": None,
+                                   "peak_source": "%s (burst bf16 matmul)" % peaks["_source"], "kernel": "attn128_ws_kernel<same head>, " + top["case"]},
+                      "gpu_launches": launches, "clocks": clocks}))
+    return 0
+
+
 def bench_merge(args):
     """vpp_lse_merge against the HBM roofline: S*(4*Dv+4) bytes read + (2*Dv+4) written per (row, head), CUDA-event timed,
     cycling through enough distinct buffers that no launch finds its inputs in the L2."""
@@ -567,7 +607,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse", "merge"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse", "merge", "groups"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -589,6 +629,8 @@ def main():
         return bench_sparse(args)
     if args.workload == "merge":
         return bench_merge(args)
+    if args.workload == "groups":
+        return bench_groups(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,
                        desc="cfg1: Hq=4 Hkv=1 d=128, 2048 tokens as 4 chunks of 512, contiguous cache"),
           "cfg2": dict(prefixes=W.CFG2_PREFIXES, chunk=8192, hq=64, hkv=4,

@@ -10,7 +10,6 @@
 #include <mutex>
 
 #include "../../include/vpp.h"
-#include "attn_simple.cuh"
 #include "attn_mla.cuh"
 #include "attn_mla2.cuh"
 #include "attn_dsa.cuh"
@@ -86,7 +85,8 @@ EncodeFn get_encode() {
 
 // Encoded tensor maps are cached: a serving loop calls with the same buffers and shapes again and again, and seven
 // to nine driver encodes per call are a visible part of a short launch.  A map depends only on (base address, rank,
-// extents, strides, box), so an entry never goes stale; the cache is a small direct-mapped table guarded by a mutex.
+// extents, strides, box), so an entry never goes stale; the cache is a small 4-way set-associative table (least recently
+// used way replaced) guarded by a mutex.
 struct TmapKey {
     const void* base;
     uint64_t dims[5];
@@ -98,23 +98,32 @@ using RawEncodeFn = bool (*)(CUtensorMap*, const TmapKey&);
 
 class TmapCache {
 public:
-    static constexpr int kSlots = 256;
+    static constexpr int kSets = 64, kWays = 4;   // a call uses up to nine maps; 256 entries serve a few dozen distinct launches
     bool get(const TmapKey& key, RawEncodeFn encode, CUtensorMap* out) {
         const uint64_t h = hash(key);
-        Slot& sl = slots_[h % kSlots];
+        Slot* set = slots_ + (h % kSets) * kWays;
         std::lock_guard<std::mutex> lk(mu_);
         ++lookups_;
-        if (sl.valid && sl.hash == h && std::memcmp(&sl.key, &key, sizeof key) == 0) {
-            *out = sl.map;
-            return true;
+        ++clock_;
+        Slot* victim = set;
+        for (int w = 0; w < kWays; ++w) {
+            Slot& sl = set[w];
+            if (sl.valid && sl.hash == h && std::memcmp(&sl.key, &key, sizeof key) == 0) {
+                sl.stamp = clock_;
+                *out = sl.map;
+                return true;
+            }
+            // the way to replace on a miss: an empty one if there is any, else the least recently used
+            if (victim->valid && (!sl.valid || sl.stamp < victim->stamp)) victim = &sl;
         }
         CUtensorMap m;
         if (!encode(&m, key)) return false;
         ++encodes_;
-        sl.key = key;
-        sl.hash = h;
-        sl.map = m;
-        sl.valid = true;
+        victim->key = key;
+        victim->hash = h;
+        victim->map = m;
+        victim->valid = true;
+        victim->stamp = clock_;
         *out = m;
         return true;
     }
@@ -126,7 +135,7 @@ public:
 private:
     struct Slot {
         TmapKey key;
-        uint64_t hash = 0;
+        uint64_t hash = 0, stamp = 0;
         CUtensorMap map;
         bool valid = false;
     };
@@ -137,8 +146,9 @@ private:
         return h;
     }
     std::mutex mu_;
-    Slot slots_[kSlots];
+    Slot slots_[kSets * kWays];
     int64_t lookups_ = 0, encodes_ = 0;
+    uint64_t clock_ = 0;
 };
 TmapCache g_tmaps;
 
@@ -297,9 +307,9 @@ int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
     return static_cast<int>(s);
 }
 
-// The pipelined kernel pairs two q-heads of one kv-head per work item; odd group sizes (MHA) take the
-// straight-line kernel, one head per item.
-bool use_ws_kernel(const vpp_chunk_attn_args* a) { return (a->num_q_heads / a->num_kv_heads) % 2 == 0; }
+// The d = 128 kernel pairs two q-heads of one kv-head per work item; when a kv-head's group is odd (MHA included) an
+// item is two consecutive 128-row query tiles of one q-head instead (work units of 256 rows).
+bool pairs_two_heads(const vpp_chunk_attn_args* a) { return (a->num_q_heads / a->num_kv_heads) % 2 == 0; }
 // The pair-of-SMs MLA kernel needs every 64-key group of a KV tile inside one page; smaller pages take the
 // single-CTA two-pass kernel.
 bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
@@ -307,7 +317,7 @@ bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
 }
 int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     if (fam == Family::kMla576) return 1;
-    return use_ws_kernel(a) ? 2 : 1;
+    return pairs_two_heads(a) ? 2 : 1;
 }
 
 using MergeKernel = void (*)(const float*, const float*, int, long long, int, int, const int32_t*, __nv_bfloat16*, float*);
@@ -550,6 +560,7 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
     pp.max_units = L.max_units;
     pp.max_cost = (a->max_seq_len + vpp::kTileN - 1) / vpp::kTileN;
     if (pp.max_cost < 1) pp.max_cost = 1;
+    pp.tile_m = (fam == Family::kGqa128 && !pairs_two_heads(a)) ? 2 * vpp::kTileM : vpp::kTileM;
     pp.partial = range ? 1 : 0;
     pp.range_begin = range ? range->begin_tile : 0;
     pp.range_end = range ? range->end_tile : 0;
@@ -592,8 +603,8 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
         if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, tm_k4, tm_k5, ap, box_rows);
-    } else if (use_ws_kernel(a)) {
-        auto kern = vpp::attn128_ws_kernel;
+    } else {
+        auto kern = pairs_two_heads(a) ? vpp::attn128_ws_kernel<false> : vpp::attn128_ws_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
         if (ce == cudaSuccess) {
             // programmatic dependent launch: set-up overlaps the work-decomposition kernel (the kernel waits for it
@@ -610,10 +621,6 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
             cfg.numAttrs = 1;
             ce = cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_v, tm_q2, tm_k2, tm_v2, tm_qh, ap, box_rows);
         }
-    } else {
-        auto kern = vpp::attn128_simple_kernel<true>;
-        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kSimpleSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kSimpleThreads, vpp::kSimpleSmemBytes, stream>>>(tm_q, tm_k, tm_v, ap, box_rows);
     }
     if (ce != cudaSuccess) return fail(VPP_ERR_CUDA, "attention kernel attributes: %s", cudaGetErrorString(ce));
     ++g_launches;

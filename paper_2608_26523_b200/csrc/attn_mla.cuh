@@ -18,7 +18,7 @@
 //   warps 2-5   softmax: one query row per thread on a 128 x 64 score tile, P written over S as bf16.
 // Tensor memory: S0 (64 cols) | S1 (64) | O half (256).
 #pragma once
-#include "attn_simple.cuh"  // decode_item
+#include "common.cuh"  // decode_item
 #include "common.cuh"
 #include "ptx.cuh"
 

@@ -1,13 +1,13 @@
-// Warp-specialised persistent chunked-prefill attention kernel for head_dim 128 (GQA / MQA with an
-// even group size).
+// Warp-specialised persistent chunked-prefill attention kernel for head_dim 128 (MHA / GQA / MQA).
 //
 // One CTA per SM, 12 warps:
 //   warp 0      scheduler + TMA producer: pops work items from the global counter, publishes them in a
 //               2-deep shared ring, loads the two Q tiles of the item and streams K/V pages through a
 //               ring of 128B-swizzled 32 KB stages (K0 V0 K1 V1 ...), gathered through the block table.
 //   warp 1      MMA issuer: tcgen05.mma  S_t = Q_t K^T  and  O_t += P_t V  for the two query tiles
-//               t = 0, 1 of the item (two q-heads of one kv-head over the same 128 query tokens, so
-//               both tiles use the same K/V stages and the same causal structure).
+//               t = 0, 1 of the item: two q-heads of one kv-head over the same 128 query tokens (even
+//               group sizes) or, when a kv-head's group is odd (MHA included), two consecutive 128-row
+//               tiles of ONE q-head -- either way both tiles use the same K/V stages.
 //   warp 2      tensor-memory allocation.
 //   warps 4-7   softmax group for tile 0: one query row per thread, fp32 online softmax on S_0 read
 //               from tensor memory, P_0 written back to tensor memory as bf16 over S_0.
@@ -25,7 +25,6 @@
 #pragma once
 #include <type_traits>
 
-#include "attn_simple.cuh"  // decode_item, kSlabBytes
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -107,11 +106,17 @@ __device__ __noinline__ void ws_packed_merge(void* out, float* lse_out, float* o
     }
 }
 
+template <bool kSameHead>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_q2,
                   const __grid_constant__ CUtensorMap tm_k2, const __grid_constant__ CUtensorMap tm_v2,
                   const __grid_constant__ CUtensorMap tm_qh, const AttnParams p, const int kv_box_rows) {
+    constexpr bool same_head = kSameHead;
+    // same_head: an item is two consecutive 128-row query tiles of one q-head (work units of up to 256 rows) instead of
+    // two q-heads over the same 128 rows -- for odd group sizes, where two q-heads need not share a kv-head.  Tile 1 then
+    // starts 128 rows (and positions) after tile 0; the KV range of the unit covers tile 1, and the causal mask hides
+    // from tile 0 what lies beyond its own rows.
     // tm_qh: the q tensor with a box of (64 features, G heads, 1 token): the rows of a packed item's Q tile
     // tm_q2 / tm_k2 / tm_v2 are views of the same tensors with the 128 features split into (64, 2): one box
     // of them brings both 64-column slabs of a 128-row tile, i.e. a whole tile per copy instruction.  Issuing a
@@ -196,7 +201,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // end of the list, which run packed when a kv-head's group fits a tile.
     const int num_packed = G <= kTileM ? p.header_ro->num_single : 0;
     const int num_normal = num_units - num_packed;
-    const int normal_items = num_normal * (p.num_q_heads / 2);
+    const int heads_per_item = same_head ? 1 : 2;
+    const int normal_items = num_normal * (p.num_q_heads / heads_per_item);
     const int total_items = normal_items + num_packed * p.num_kv_heads;
 
     if (warp < 4) {
@@ -213,9 +219,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 bool packed = false;
                 if (have && item < normal_items) {
                     int ui, hp;
-                    decode_item(item, num_normal, p.num_q_heads / 2, G / 2, ui, hp);
+                    decode_item(item, num_normal, p.num_q_heads / heads_per_item, G / heads_per_item, ui, hp);
                     u = p.units[ui];
-                    h0 = 2 * hp;
+                    h0 = heads_per_item * hp;
                 } else if (have) {
                     const int k = item - normal_items;
                     u = p.units[num_normal + k / p.num_kv_heads];
@@ -248,7 +254,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     } else if (ok) {
                         mbar_arrive_expect_tx(bar_q_full, 2 * kTileBytes);
                         tma_load_4d(sQ, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0);
-                        tma_load_4d(sQ + kTileBytes, &tm_q2, bar_q_full, 0, u.q_row0, 0, h0 + 1);
+                        // (rows past the end of q read as zero; rows of a following request are never stored)
+                        tma_load_4d(sQ + kTileBytes, &tm_q2, bar_q_full, 0, u.q_row0 + (same_head ? kTileM : 0), 0,
+                                    h0 + (same_head ? 0 : 1));
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -526,7 +534,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             if (!mbar_wait(bar_item_full + 8 * slot, (item_it >> 1) & 1, s_abort, 401)) break;
             const WorkUnit u = ring[slot].u;
             const bool packed = ring[slot].packed != 0;
-            const int h = ring[slot].h0 + (packed ? row : t);   // packed: row r of tile 0 is q-head h0 + r
+            // packed: row r of tile 0 is q-head h0 + r; otherwise tile t is q-head h0 + t, or rows 128 t .. of q-head h0
+            const int h = ring[slot].h0 + (packed ? row : (same_head ? 0 : t));
+            const int row_base = (!packed && same_head) ? t * kTileM : 0;
             const int valid = ring[slot].valid;
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
@@ -538,10 +548,11 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             constexpr bool kPacked = decltype(packed_tag)::value;
             // rows of this thread's warp that exist: a packed tile has G rows, a warp without any only keeps the
             // barriers moving
-            const int tile_rows = kPacked ? G : u.rows;
+            const int tile_rows = kPacked ? G : u.rows - row_base;   // (<= 0: tile 1 of a unit of at most 128 rows is idle)
             const bool warp_idle = kPacked && (warp & 3) * 32 >= G;
 
-            const int my_pos = kPacked ? u.pos0 : u.pos0 + row;
+            const int tile_pos0 = u.pos0 + row_base;               // position of the tile's first row
+            const int my_pos = kPacked ? u.pos0 : tile_pos0 + row;
             float m_ref = -INFINITY, l_run = 0.f;
             bool ok = true;
             // a packed item: this group's tile takes every second KV tile
@@ -561,7 +572,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     continue;
                 }
                 uint32_t s[128];
-                const bool diag = tile0 + kTileN - 1 > u.pos0;  // keys beyond the row's position are masked
+                const bool diag = tile0 + kTileN - 1 > tile_pos0;  // keys beyond the row's position are masked
                 const int lim = my_pos - tile0;                 // columns <= lim are visible
                 float mx[8];
                 // the second half of the row is still in flight while the first half is reduced
@@ -675,7 +686,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             {
                 const float inv_l = 1.f / l_run;
                 const bool live = row < tile_rows;
-                const long long grow_idx = static_cast<long long>(u.q_row0) + row;
+                const long long grow_idx = static_cast<long long>(u.q_row0) + row_base + row;
                 uint32_t r[32];
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {

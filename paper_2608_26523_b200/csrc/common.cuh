@@ -13,7 +13,7 @@ constexpr int kTileN = 128;  // keys per KV tile
 struct __align__(16) WorkUnit {
     int32_t req;        // request index
     int32_t q_row0;     // first packed query row of the tile
-    int32_t rows;       // valid rows in the tile (1..128)
+    int32_t rows;       // valid rows in the unit (1..128; up to 256 when an item is two tiles of one q-head)
     int32_t pos0;       // absolute position of the tile's first row (prefix_len + row offset)
     int32_t kv_begin;   // first KV tile (units of kTileN keys)
     int32_t kv_end;     // one past the last KV tile
@@ -58,5 +58,25 @@ struct AttnParams {
     const WorkUnit* units;
     int32_t* status;              // may be null
 };
+
+constexpr int kSlabBytes = kTileM * 128;  // 128 rows x 64 bf16, 128B-swizzled
+
+// Which (unit, kv-head, q-head) a flat work index means.  Units arrive sorted by decreasing cost; inside
+// a block of kUnitBlock consecutive units the items are ordered kv-head-major so that CTAs running at
+// the same time read the same K/V pages (L2 reuse), while blocks keep the longest-first order.
+constexpr int kUnitBlock = 32;
+__device__ __forceinline__ void decode_item(int w, int num_units, int items_per_unit, int per_kv_head, int& unit,
+                                            int& slot) {
+    const int blk_items = kUnitBlock * items_per_unit;
+    const int ub = w / blk_items;
+    const int rem = w - ub * blk_items;
+    const int left = num_units - ub * kUnitBlock;
+    const int nblk = left < kUnitBlock ? left : kUnitBlock;
+    const int per_g = nblk * per_kv_head;
+    const int g = rem / per_g;
+    const int rem2 = rem - g * per_g;
+    unit = ub * kUnitBlock + rem2 / per_kv_head;
+    slot = g * per_kv_head + rem2 % per_kv_head;
+}
 
 }  // namespace vpp

@@ -1,5 +1,5 @@
 // Work decomposition: from the per-request (prefix_len, chunk_len) on the device, build the list of
-// work units (128-row query tile x key-range split) ordered by decreasing cost, so that the
+// work units (query tile of 128 -- or 256 -- rows x key-range split) ordered by decreasing cost, so that the
 // persistent attention kernel can hand out tiles of very unequal cost longest-first.
 //
 // A query tile whose first row sits at absolute position pos0 needs the KV tiles
@@ -27,6 +27,7 @@ struct PrepParams {
     int32_t splits;      // S >= 1
     int32_t max_units;
     int32_t max_cost;    // ceil(max_seq_len / 128), >= 1
+    int32_t tile_m;      // query rows per unit: 128, or 256 when a work item is two 128-row tiles of one q-head
     int32_t partial;     // 1: key-range restricted launch whose results are partial (o fp32, lse) of "split 0"
     int32_t range_begin; // first KV tile of the key range (partial launches)
     int32_t range_end;   // one past its last KV tile
@@ -115,7 +116,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
                 atomicExch(&s_error, 1 /* VPP_DEV_BAD_LENGTHS */);
                 c = 0;
             }
-            nt = (c + kTileM - 1) / kTileM;
+            nt = (c + p.tile_m - 1) / p.tile_m;
         }
         int tot_q, tot_t;
         const int eq = block_exclusive_scan(c, warp_sums, tot_q);
@@ -179,8 +180,8 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
             const int r = lo;
             const int qt = gt - p.tile_start[r];
             const int P = p.prefix_len[r], C = p.chunk_len[r];
-            const int row_off = qt * kTileM;
-            const int rows = (C - row_off) < kTileM ? (C - row_off) : kTileM;
+            const int row_off = qt * p.tile_m;
+            const int rows = (C - row_off) < p.tile_m ? (C - row_off) : p.tile_m;
             const int pos0 = P + row_off;
             const int n_tiles = (pos0 + rows + kTileN - 1) / kTileN;
             const int nsplit = p.partial ? 1 : tile_num_splits(pos0, p.splits);
