@@ -160,3 +160,30 @@ def test_host_streaming_pipeline_with_planned_slices():
     assert int(pipe.status.max().item()) == 0
     rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
     print(plan, compare(out_host, lse_host, prob_cpu, rows, "planned slices"))
+
+
+def test_host_streaming_pipeline_at_benchmark_size_matches_the_oracle():
+    """The end-to-end leg of bench.py at its real size: the cfg 2 chunk at prefix 65536 streamed from pinned host memory in
+    the planned slices, compared with the oracle on one row of every (query tile, pair of q-heads) plus the edge rows."""
+    from parity import sample_rows, tile_rows
+    prob = W.cfg2(prefix=65536, device="cuda")
+    prob_cpu = prob.to("cpu")
+    pipe = api.HostChunkPipeline(prob)
+    q_host = prob_cpu.q.clone().pin_memory()
+    blocks = pipe.chunk_blocks()
+    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
+    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
+    prob.q.fill_(float("nan"))                      # what the pipeline brings in is not on the device beforehand
+    for b in blocks:
+        prob.k_cache[b] = float("nan")
+        prob.v_cache[b] = float("nan")
+    out_host = torch.full((8192, 64, 128), float("nan"), dtype=torch.bfloat16).pin_memory()
+    lse_host = torch.full((8192, 64), float("nan"), dtype=torch.float32).pin_memory()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+    stream.synchronize()
+    assert int(pipe.status.max().item()) == 0
+    assert torch.isfinite(out_host.float()).all() and torch.isfinite(lse_host).all()
+    rows = np.unique(np.concatenate([sample_rows(prob_cpu, n_random=64), tile_rows(prob_cpu, per="pair", seed=3)]), axis=0)
+    print(compare(out_host, lse_host, prob_cpu, rows, "host pipeline, cfg2 at 65536"))
