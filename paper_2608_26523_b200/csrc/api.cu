@@ -570,7 +570,14 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
     pp.q_start = row_splits + a->total_q;
     pp.tile_start = pp.q_start + a->num_reqs + 1;
     pp.status = a->status;
-    vpp::prep_kernel<<<1, vpp::kPrepThreads, 0, stream>>>(pp);
+    {
+        // small launches (a short chunk, a small decode batch) take the one-warp decomposition
+        const long long tiles_ub = (a->total_q + pp.tile_m - 1) / pp.tile_m + a->num_reqs;
+        if (a->num_reqs <= vpp::kPrepSmallMax && tiles_ub <= vpp::kPrepSmallMax)
+            vpp::prep_small_kernel<<<1, 32, 0, stream>>>(pp);
+        else
+            vpp::prep_kernel<<<1, vpp::kPrepThreads, 0, stream>>>(pp);
+    }
     ++g_launches;
 
     // ---- attention ----

@@ -244,4 +244,142 @@ __global__ void __launch_bounds__(kPrepThreads, 1) prep_kernel(const PrepParams 
     }
 }
 
+// The same decomposition for small launches (at most 32 requests and 32 query tiles: a short chunk, a small decode
+// batch), by ONE warp: a lane per request, then a lane per query tile, scans by shuffles, no block-wide
+// synchronisation, no sort -- the units of such a launch all start in the first wave of work items, so their order
+// does not matter (units of several rows first, single-token units last, as the attention kernels expect).  About a
+// third of the big kernel's latency, which is most of what a launch of a few work items costs.
+constexpr int kPrepSmallMax = 32;
+
+__global__ void __launch_bounds__(32, 1) prep_small_kernel(const PrepParams p) {
+    __shared__ int s_P[kPrepSmallMax], s_C[kPrepSmallMax], s_q0[kPrepSmallMax + 1], s_t0[kPrepSmallMax + 1];
+    const int lane = threadIdx.x;
+    pdl_launch_dependents();
+    // ---- requests: validate, scan chunk lengths and tile counts ----
+    int P = 0, c = 0, nt = 0, bad = 0;
+    if (lane < p.num_reqs) {
+        P = p.prefix_len[lane];
+        c = p.chunk_len[lane];
+        if (P < 0 || c < 0 || static_cast<long long>(P) + c > p.max_seq_len ||
+            (p.partial && c > 0 && P < p.range_begin * kTileN)) {
+            bad = 1;
+            c = 0;
+        }
+        nt = (c + p.tile_m - 1) / p.tile_m;
+    }
+    int iq = c, it = nt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, iq, o), b = __shfl_up_sync(0xffffffffu, it, o);
+        if (lane >= o) {
+            iq += a;
+            it += b;
+        }
+    }
+    const int total_q = __shfl_sync(0xffffffffu, iq, 31), total_tiles = __shfl_sync(0xffffffffu, it, 31);
+    if (lane < p.num_reqs) {
+        s_P[lane] = P;
+        s_C[lane] = c;
+        s_q0[lane] = iq - c;
+        s_t0[lane] = it - nt;
+        p.q_start[lane] = iq - c;
+        p.tile_start[lane] = it - nt;
+    }
+    if (lane == 0) {
+        s_t0[p.num_reqs] = total_tiles;
+        p.q_start[p.num_reqs] = total_q;
+        p.tile_start[p.num_reqs] = total_tiles;
+    }
+    int error = __any_sync(0xffffffffu, bad) || total_q != p.total_q || total_tiles > kPrepSmallMax ? 1 : 0;
+    __syncwarp();
+    // ---- every block-table entry a request needs must name a real block ----
+    if (error == 0 && p.block_table != nullptr) {
+        int bad_blk = 0;
+        for (int r = 0; r < p.num_reqs; ++r) {
+            if (s_C[r] == 0) continue;
+            const int nb = (s_P[r] + s_C[r] + (1 << p.block_shift) - 1) >> p.block_shift;
+            if (nb > p.max_blocks_per_req) {
+                bad_blk = 1;
+                continue;
+            }
+            for (int b = lane; b < nb; b += 32) {
+                const int e = p.block_table[static_cast<long long>(r) * p.max_blocks_per_req + b];
+                if (e < 0 || e >= p.num_blocks) bad_blk = 1;
+            }
+        }
+        if (__any_sync(0xffffffffu, bad_blk)) error = 2;
+    }
+    if (error != 0) {
+        if (lane == 0) {
+            p.header->num_units = 0;
+            p.header->num_single = 0;
+            p.header->counter = 0;
+            p.header->error = error;
+            if (p.status) *p.status = error;
+        }
+        return;
+    }
+    // ---- a lane per query tile: its units, placed by two scans (units of several rows, then single-token units) ----
+    int r = 0, rows = 0, pos0 = 0, n_tiles = 0, nsplit = 0, row_off = 0;
+    if (lane < total_tiles) {
+        while (s_t0[r + 1] <= lane) ++r;
+        row_off = (lane - s_t0[r]) * p.tile_m;
+        rows = s_C[r] - row_off < p.tile_m ? s_C[r] - row_off : p.tile_m;
+        pos0 = s_P[r] + row_off;
+        n_tiles = (pos0 + rows + kTileN - 1) / kTileN;
+        nsplit = p.partial ? 1 : tile_num_splits(pos0, p.splits);
+    }
+    const bool single = rows == 1;
+    int in = single ? 0 : nsplit, is = single ? nsplit : 0;
+    const int mine_n = in, mine_s = is;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, in, o), b = __shfl_up_sync(0xffffffffu, is, o);
+        if (lane >= o) {
+            in += a;
+            is += b;
+        }
+    }
+    const int total_n = __shfl_sync(0xffffffffu, in, 31), total_s = __shfl_sync(0xffffffffu, is, 31);
+    const int first = single ? total_n + is - mine_s : in - mine_n;
+    for (int s = 0; s < nsplit; ++s) {
+        int kb, ke;
+        if (p.partial) {
+            kb = p.range_begin;
+            ke = n_tiles < p.range_end ? n_tiles : p.range_end;
+        } else {
+            split_range(pos0, n_tiles, nsplit, s, kb, ke);
+        }
+        if (first + s < p.max_units) {
+            WorkUnit u;
+            u.req = r;
+            u.q_row0 = s_q0[r] + row_off;
+            u.rows = rows;
+            u.pos0 = pos0;
+            u.kv_begin = kb;
+            u.kv_end = ke;
+            u.split = (nsplit > 1 || p.partial) ? s : -1;
+            u.kv_len = s_P[r] + s_C[r];
+            p.units[first + s] = u;
+        }
+    }
+    if (p.splits > 1) {
+        // per-row split counts, written by the whole warp tile by tile
+        for (int t = 0; t < total_tiles; ++t) {
+            const int t_rows = __shfl_sync(0xffffffffu, rows, t), t_ns = __shfl_sync(0xffffffffu, nsplit, t);
+            const int t_q0 = __shfl_sync(0xffffffffu, lane < total_tiles ? s_q0[r] + row_off : 0, t);
+            for (int i = lane; i < t_rows; i += 32) p.row_splits[t_q0 + i] = t_ns;
+        }
+    }
+    if (lane == 0) {
+        const int n = total_n + total_s < p.max_units ? total_n + total_s : p.max_units;
+        const int first_single = total_n < n ? total_n : n;
+        p.header->num_units = n;
+        p.header->num_single = n - first_single;
+        p.header->counter = 0;
+        p.header->error = 0;
+        if (p.status) *p.status = 0;
+    }
+}
+
 }  // namespace vpp
