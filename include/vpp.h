@@ -275,7 +275,8 @@ vpp_status vpp_kv_append(const vpp_kv_append_args *args, vpp_stream_t stream);
  * q            bf16 [total_q, num_q_heads, 576], dense, packed request-major. 16-byte aligned. num_q_heads <= 128.
  * kv_cache     bf16 latent cache, one kv-head of 576 features per position; values are features 0..511 of the same
  *              row.  Position pos of request r is row block_table[r][pos / block_size] * block_size + pos % block_size
- *              (block_table NULL: r * max_seq_len + pos); rows are kv_row_stride elements apart (a multiple of 8,
+ *              (block_table NULL: r * max_seq_len + pos, so the cache must hold num_reqs * max_seq_len rows); rows are
+ *              kv_row_stride elements apart (a multiple of 8,
  *              >= 576), so a paged cache must have block stride = block_size * row stride.  16-byte aligned.  The
  *              cache must hold the chunk's own positions (every token's own row is read).
  * indices      int32 [total_q, topk], topk >= 1.

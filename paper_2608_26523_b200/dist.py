@@ -69,10 +69,18 @@ def partition_requests(prefix_lens, chunk_lens, world):
     return [sorted(x) for x in parts]
 
 
-def kv_ranges(seq_len, world):
-    """Contiguous, 128-aligned KV ranges [lo, hi) of a context-parallel split of one sequence."""
+def kv_ranges(seq_len, world, prefix_len=None):
+    """Contiguous, 128-aligned KV ranges [lo, hi) of a context-parallel split of one sequence.
+
+    With prefix_len (the tokens cached before the current chunk) no range starts beyond the prefix, which is what
+    vpp_chunk_attn_partial_fwd needs (every query row must see a key of every range): the chunk's own keys stay with the
+    last range.  Ranges may be empty (lo == hi) when there are more ranks than 128-key tiles; an empty range is skipped
+    by its rank (its partial is lse = -inf)."""
     tiles = (seq_len + 127) // 128
     cuts = [min(seq_len, ((tiles * r) // world) * 128) for r in range(world)] + [seq_len]
+    if prefix_len is not None:
+        cap = (int(prefix_len) // 128) * 128
+        cuts = [min(c, cap) for c in cuts[:-1]] + [seq_len]
     return [(cuts[r], cuts[r + 1]) for r in range(world)]
 
 

@@ -100,3 +100,10 @@ def test_kv_ranges_cover_the_sequence():
         r = D.kv_ranges(n, w)
         assert r[0][0] == 0 and r[-1][1] == n and all(a[1] == b[0] for a, b in zip(r, r[1:]))
         assert all(lo % 128 == 0 for lo, _ in r)
+
+
+def test_kv_ranges_with_a_prefix_start_inside_it():
+    for seq, pre, w in [(5700, 5000, 4), (900, 130, 4), (700, 0, 2), (100000, 99000, 8)]:
+        r = D.kv_ranges(seq, w, prefix_len=pre)
+        assert r[0][0] == 0 and r[-1][1] == seq and all(a[1] == b[0] for a, b in zip(r, r[1:]))
+        assert all(lo % 128 == 0 and lo <= pre for lo, _ in r)

@@ -116,3 +116,26 @@ def test_a_key_range_beyond_a_request_prefix_is_refused_on_the_device():
     torch.cuda.synchronize()
     assert int(runner.status.item()) == 1                                 # VPP_DEV_BAD_LENGTHS
     assert (o == 7.0).all() and (l == 7.0).all()                          # nothing written
+
+
+@pytest.mark.parametrize("world", [2, 4])
+@pytest.mark.parametrize("mla", [False, True])
+def test_context_parallel_ranks_emulated_on_one_gpu(world, mla):
+    """The KV-range split of dist.kv_ranges with the library as every rank's kernel: rank r's launch sees only its range of
+    the cache, the partials are stacked as an all-gather would stack them and merged.  (One GPU: the ranks run in turn.)"""
+    from paper_2608_26523_b200 import dist as D
+    if mla:
+        prob = W.make_problem(51, [3000], [450], 16, 1, 576, 512, block_size=64, std=0.5, v_aliases_k=True)
+    else:
+        prob = W.make_problem(52, [5000], [700], 8, 2, 128, 128, block_size=128)
+    P, C = int(prob.prefix_len[0]), int(prob.chunk_len[0])
+    ranges = [(lo, hi) for lo, hi in D.kv_ranges(P + C, world, prefix_len=P) if hi > lo]
+    assert len(ranges) == world
+    gpu = prob.to("cuda")
+    runner, o_parts, lse_parts = _partials(gpu, ranges)
+    out = torch.empty((gpu.total_q, gpu.num_q_heads, gpu.head_dim_v), dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty((gpu.total_q, gpu.num_q_heads), dtype=torch.float32, device="cuda")
+    api.vpp_lse_merge(o_parts, lse_parts, out, lse)
+    torch.cuda.synchronize()
+    rows = oracle.all_rows(prob.chunk_len.numpy(), prob.num_q_heads)
+    print(compare(out, lse, prob, rows, "context parallel, %d ranks" % world))

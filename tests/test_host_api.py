@@ -268,3 +268,21 @@ def test_bounded_wait_hook_checks_its_arguments(lib):
     st = torch.zeros(1, dtype=torch.int32)
     assert lib.vpp_test_bounded_wait(st.data_ptr(), 0, None) == api.VPP_ERR_INVALID_ARG
     assert lib.vpp_test_bounded_wait(st.data_ptr(), 1 << 40, None) == api.VPP_ERR_INVALID_ARG
+
+
+def test_cost_curve_fit_and_balance_identity_of_the_benchmark():
+    """bench.py's evaluation of the paper's Eq. 2 (affine latency) and Eq. 3 (tau(k-1) + tau(k+1) = 2 tau(k)) on a measured
+    curve: exact on an affine curve, and the residual of a known bend on the evenly spaced triples only."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    xs = [0, 8192, 32768, 65536, 98304, 131072]
+    fit = bench.fit_cost_curve(xs, [1.0 + 2e-4 * x for x in xs])
+    assert abs(fit["fit_ms"]["a"] - 1.0) < 1e-4 and abs(fit["fit_ms"]["b_per_token"] - 2e-4) < 1e-9
+    assert fit["eq3_residual_max"] < 1e-9 and fit["eq3_triples"] == 4      # (0,32K,64K) (32K,64K,96K) (64K,96K,128K) (0,64K,128K)
+    bent = bench.fit_cost_curve([0, 100, 200], [1.0, 2.0, 4.0])
+    assert abs(bent["eq3_residual_max"] - abs(1.0 + 4.0 - 4.0) / 4.0) < 1e-4
+    assert bench.fit_cost_curve([0, 100], [1.0, 2.0]) is None
+    rec = bench.read_traffic_record("attn128_ws_cfg2_traffic.txt")
+    assert rec["prefix"] == "131072" and float(rec["dram_bytes_read"]) > 0 and rec["kernel"] == "attn128_ws_kernel"
