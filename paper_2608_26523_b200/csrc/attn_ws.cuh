@@ -31,6 +31,12 @@
 namespace vpp {
 
 constexpr int kWsThreads = 384;
+// Register budget per thread after the roles split (setmaxnreg).  The launch gives every warp 168 registers (three warps
+// per sub-partition); warps 0-3 (one per sub-partition: producer, MMA issuer, allocator, idle) hand back down to
+// kWsRegsLow and each of the two softmax warps of a sub-partition takes kWsRegsHigh: 72 + 2 * 216 = 3 * 168.  With 216
+// registers the softmax loop (128 scores of a row live at once) has no spills.
+constexpr int kWsRegsLow = 72, kWsRegsHigh = 216;
+static_assert(kWsRegsLow + 2 * kWsRegsHigh <= 3 * 168 && kWsRegsLow % 8 == 0 && kWsRegsHigh % 8 == 0, "register budget");
 constexpr int kWsStages = 4;                  // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 2048 /*barriers, ring, merge exchange*/;
@@ -206,6 +212,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int total_items = normal_items + num_packed * p.num_kv_heads;
 
     if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kWsRegsLow));
         if (warp == 0) {
             // ============================ scheduler + TMA producer ============================
             uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_cnt = 0;
@@ -521,6 +528,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // warps 2 and 3 have nothing to do until teardown
     } else {
         // ===================================== softmax groups =====================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kWsRegsHigh));
         const int t = (warp - 4) >> 2;                 // query tile / softmax group
         const int row = ((warp & 3) << 5) | lane;      // row of the tile = TMEM lane
         const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
