@@ -760,32 +760,23 @@ def main():
             i_main = prefixes.index(65536) if 65536 in prefixes else len(prefixes) - 1
             r = runners[i_main]
             P = prefixes[i_main]
+            # The public call for host-resident inputs, vpp_chunk_attn_host_fwd: q and the chunk's own K/V rows come from
+            # pinned host memory, out and lse go back to it; the library streams the chunk in slices, the copies of one
+            # slice overlapping the append + attention of its neighbours.  Every step copies all inputs in and all
+            # results out, and no step starts before the previous one's last copy has finished.
+            slices = None if args.e2e_slices == "auto" else [int(x) for x in args.e2e_slices.split(",")]
+            pipe = api.HostChunkPipeline(r.prob, slices=slices, num_kv_splits=args.splits)
+            e2e_plan = pipe.slices
             q_host = r.prob.q.cpu().pin_memory()
+            k_host = pipe.chunk_rows(r.prob.k_cache).cpu().contiguous().pin_memory()
+            v_host = pipe.chunk_rows(r.prob.v_cache).cpu().contiguous().pin_memory()
             out_host = torch.empty(r.out.shape, dtype=r.out.dtype).pin_memory()
             lse_host = torch.empty(r.lse.shape, dtype=r.lse.dtype).pin_memory()
-            bt = r.prob.block_table[0].cpu().tolist()
-            B = r.prob.block_size
-            chunk_blocks = [bt[j] for j in range(P // B, (P + chunk + B - 1) // B)]
-            k_host = [r.prob.k_cache[b].cpu().pin_memory() for b in chunk_blocks]
-            v_host = [r.prob.v_cache[b].cpu().pin_memory() for b in chunk_blocks]
-            h2d = q_host.numel() * 2 + sum(t.numel() * 2 for t in k_host + v_host)
+            h2d = (q_host.numel() + k_host.numel() + v_host.numel()) * 2
             d2h = out_host.numel() * 2 + lse_host.numel() * 4
 
-            # The public call for host-resident inputs: the chunk streamed in slices, copies of one slice
-            # overlapping the attention of its neighbours (api.HostChunkPipeline); every step copies all inputs in and
-            # all results out, and no step starts before the previous one's last copy has finished.
-            if args.e2e_slices == "auto":
-                pipe = api.HostChunkPipeline(r.prob, slices="auto", num_kv_splits=args.splits)
-            else:
-                e2e_slices = [int(x) for x in args.e2e_slices.split(",")]
-                pipe = api.HostChunkPipeline(r.prob, slices=e2e_slices[0] if len(e2e_slices) == 1 else e2e_slices,
-                                             num_kv_splits=args.splits)
-            e2e_plan = [hi - lo for (lo, hi, *_rest) in pipe.parts]
-            k_pages = dict(zip(chunk_blocks, k_host))
-            v_pages = dict(zip(chunk_blocks, v_host))
-
             def e2e_step():
-                pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+                pipe.run(q_host, k_host, v_host, out_host, lse_host, stream)
 
             for _ in range(2):
                 e2e_step()
@@ -800,7 +791,7 @@ def main():
             e2e_ms = t0.elapsed_time(t1) / n_e2e
             e2e = (flops_pt[i_main], e2e_ms, h2d, d2h, P)
             # the streamed result is the resident launch's result
-            assert int(pipe.status.max().item()) == 0
+            assert int(pipe.status.item()) == 0
             r.run(stream.cuda_stream)
             stream.synchronize()
             diff = (out_host[::7].float() - r.out[::7].float().cpu()).abs().max().item()
@@ -869,8 +860,9 @@ def main():
         line["e2e"] = {"value": round(world * e2e[0] / (e2e[1] * 1e-3) / 1e12, 3), "unit": UNIT,
                        "h2d_bytes_per_step": int(e2e[2]), "d2h_bytes_per_step": int(e2e[3]),
                        "ms_per_step": round(e2e[1], 4),
-                       "workload": "the chunk at prefix %d: q and the chunk's K/V pages host->device, out and lse device->host, "
-                                   "streamed in slices of %s query rows whose copies overlap the neighbouring slices' attention" % (e2e[4], e2e_plan)}
+                       "workload": "vpp_chunk_attn_host_fwd on the chunk at prefix %d: q and the chunk's K/V rows host->device, "
+                                   "appended to the cache, out and lse device->host, streamed in slices of %s query rows whose "
+                                   "copies overlap the neighbouring slices' append + attention" % (e2e[4], e2e_plan)}
     if not args.no_cpu_baseline and world == 1 and args.workload == "cfg2":
         prob_cpu = runners[prefixes.index(65536) if 65536 in prefixes else -1].prob.to("cpu")
         fl, dt, n, threads = oracle_sample_rate(prob_cpu, 15.0, np.random.default_rng(0))
@@ -880,7 +872,7 @@ def main():
     if args.workload == "cfg2" and world == 1 and not args.no_sweep and not args.prefixes:
         del runners
         if e2e:
-            del pipe, q_host, out_host, lse_host, k_host, v_host, k_pages, v_pages
+            del pipe, q_host, out_host, lse_host, k_host, v_host
         base = None
         torch.cuda.empty_cache()
         line["configs"] = sweep_other_configs(dev, peaks, max(3, min(args.steps, 5)), max(3, args.warmup), not args.no_cpu_baseline)

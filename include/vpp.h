@@ -264,6 +264,64 @@ typedef struct {
 vpp_status vpp_kv_append(const vpp_kv_append_args *args, vpp_stream_t stream);
 
 /*
+ * One chunk of one request with its query, its new keys/values and its results in HOST memory: the whole per-chunk
+ * step of a chunked prefill (the paper's "Chunked Prefill Pipeline Parallelism" section: append the chunk's K/V to
+ * the cache, then Eq. 1 over prefix + chunk) as a single call that also moves the data.  The chunk's rows are cut
+ * into slices; slice i's rows go host -> device on a copy stream of the library, are appended (vpp_kv_append) and
+ * attended (vpp_chunk_attn_fwd, prefix = prefix_len + the earlier slices) on `stream`, and its results go device ->
+ * host on a second copy stream, so that the copies of a slice overlap the attention of its neighbours.  No
+ * arithmetic happens outside those two entry points' kernels.
+ *
+ * q_host       bf16 [chunk_len, num_q_heads, head_dim_qk]   host, read
+ * k_new_host   bf16 [chunk_len, num_kv_heads, head_dim_qk]  host, read: keys of the chunk's own tokens
+ * v_new_host   bf16 [chunk_len, num_kv_heads, head_dim_v]   host, read; ignored when dev.v_cache == dev.k_cache (MLA)
+ * out_host     bf16 [chunk_len, num_q_heads, head_dim_v]    host, written
+ * lse_host     float [chunk_len, num_q_heads] or NULL       host, written
+ *              Host buffers should be page-locked (copies from pageable memory do not overlap anything); they must
+ *              stay valid until the work enqueued on `stream` has completed.
+ * prefix_len, chunk_len   host scalars of the request; positions [0, prefix_len) are in the cache already.
+ * slice_rows, num_slices  slice lengths in rows (positive, sum = chunk_len, at most VPP_HOST_MAX_SLICES), or NULL / 0:
+ *              the library cuts the chunk into three runs of whole 128-row tiles that minimise what cannot overlap
+ *              (first copy in, last copy out, idle tail of each launch's last wave); chunks of fewer than three
+ *              tiles or ragged chunks go through as one slice.  vpp_chunk_attn_host_plan returns that choice.
+ * dev          the device side, as for vpp_chunk_attn_fwd with num_reqs = 1 and total_q = chunk_len: caches and
+ *              strides, block_table (device, one row), geometry, softmax_scale, num_kv_splits; q / out / lse are
+ *              DEVICE staging buffers of the chunk's size (lse may be NULL iff lse_host is NULL); prefix_len and
+ *              chunk_len are ignored (the library writes its own per slice); workspace of at least
+ *              vpp_chunk_attn_host_workspace_size bytes; status optional device int32: the first nonzero status of
+ *              the call's launches in launch order, 0 if none.  The caches are WRITTEN (the chunk's rows) and read.
+ * k_new_dev, v_new_dev    device staging for the chunk's key / value rows, sizes as k_new_host / v_new_host
+ *              (v_new_dev may be NULL under MLA aliasing).
+ * Calls on one device are enqueued one at a time (a process-wide lock) and share two copy streams and their events,
+ * created on the first call on that device (not a stream operation: make that first call outside any capture).
+ * On return everything is enqueued and `stream` waits for the last device -> host copy.  Errors: as
+ * vpp_chunk_attn_fwd and vpp_kv_append (vpp_host_last_error() has the detail); VPP_ERR_CUDA if a copy or an event
+ * operation fails -- earlier slices may have been enqueued by then.
+ */
+#define VPP_HOST_MAX_SLICES 16
+typedef struct {
+    const void *q_host;
+    const void *k_new_host;
+    const void *v_new_host;
+    void *out_host;
+    float *lse_host;
+    int32_t prefix_len;
+    int32_t chunk_len;
+    const int32_t *slice_rows;
+    int32_t num_slices;
+    vpp_chunk_attn_args dev;
+    void *k_new_dev;
+    void *v_new_dev;
+} vpp_chunk_attn_host_args;
+
+size_t vpp_chunk_attn_host_workspace_size(const vpp_chunk_attn_host_args *args);
+/* Writes the slice lengths the call would use (at most VPP_HOST_MAX_SLICES) and returns their number; 0 if invalid. */
+int32_t vpp_chunk_attn_host_plan(const vpp_chunk_attn_host_args *args, int32_t *slice_rows_out);
+vpp_status vpp_chunk_attn_host_fwd(const vpp_chunk_attn_host_args *args, vpp_stream_t stream);
+/* Thread-local detail of the last failure of the three functions above on this host thread. */
+const char *vpp_host_last_error(void);
+
+/*
  * Index-selected (sparse) chunk attention over the absorbed-MLA latent cache: the attention of the paper's third
  * model ("MLA + DSA sparse attention", evaluation set-up; its "Impact of Sparse Attention" paragraph is about the
  * flat cost curve this has).  The selection itself (a learned top-k indexer) is an input: for every query token a

@@ -22,7 +22,8 @@ EXPORTS = ["vpp_chunk_attn_workspace_size", "vpp_chunk_attn_fwd", "vpp_lse_merge
            "vpp_last_error", "vpp_last_launch_count", "vpp_chunk_attn_fwd_static", "vpp_static_scratch_bytes",
            "vpp_static_last_error", "vpp_kv_append", "vpp_sparse_attn_workspace_size", "vpp_sparse_mla_fwd",
            "vpp_chunk_attn_partial_fwd", "vpp_tensor_map_cache_stats", "vpp_test_tensor_map_cache",
-           "vpp_test_bounded_wait"]
+           "vpp_test_bounded_wait", "vpp_chunk_attn_host_workspace_size", "vpp_chunk_attn_host_plan",
+           "vpp_chunk_attn_host_fwd", "vpp_host_last_error"]
 
 
 class VppError(RuntimeError):
@@ -72,6 +73,16 @@ class SparseAttnArgs(ctypes.Structure):
     ]
 
 
+class HostChunkAttnArgs(ctypes.Structure):
+    _fields_ = [
+        ("q_host", ctypes.c_void_p), ("k_new_host", ctypes.c_void_p), ("v_new_host", ctypes.c_void_p),
+        ("out_host", ctypes.c_void_p), ("lse_host", ctypes.c_void_p),
+        ("prefix_len", ctypes.c_int32), ("chunk_len", ctypes.c_int32),
+        ("slice_rows", ctypes.c_void_p), ("num_slices", ctypes.c_int32),
+        ("dev", ChunkAttnArgs), ("k_new_dev", ctypes.c_void_p), ("v_new_dev", ctypes.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -113,6 +124,13 @@ def load_library():
         lib.vpp_test_tensor_map_cache.argtypes = [ctypes.c_int32]
         lib.vpp_test_bounded_wait.restype = ctypes.c_int
         lib.vpp_test_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+        lib.vpp_chunk_attn_host_workspace_size.restype = ctypes.c_size_t
+        lib.vpp_chunk_attn_host_workspace_size.argtypes = [ctypes.POINTER(HostChunkAttnArgs)]
+        lib.vpp_chunk_attn_host_plan.restype = ctypes.c_int32
+        lib.vpp_chunk_attn_host_plan.argtypes = [ctypes.POINTER(HostChunkAttnArgs), ctypes.POINTER(ctypes.c_int32)]
+        lib.vpp_chunk_attn_host_fwd.restype = ctypes.c_int
+        lib.vpp_chunk_attn_host_fwd.argtypes = [ctypes.POINTER(HostChunkAttnArgs), ctypes.c_void_p]
+        lib.vpp_host_last_error.restype = ctypes.c_char_p
         _lib = lib
     return _lib
 
@@ -324,103 +342,81 @@ class ChunkAttn:
         return self.out, self.lse
 
 
+def vpp_chunk_attn_host_workspace_size(hargs):
+    return int(load_library().vpp_chunk_attn_host_workspace_size(ctypes.byref(hargs)))
+
+
+def vpp_chunk_attn_host_plan(hargs):
+    rows = (ctypes.c_int32 * 16)()
+    n = int(load_library().vpp_chunk_attn_host_plan(ctypes.byref(hargs), rows))
+    return [int(rows[i]) for i in range(n)]
+
+
+def vpp_chunk_attn_host_fwd(hargs, stream=None):
+    lib = load_library()
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif hasattr(stream, "cuda_stream"):
+        stream = stream.cuda_stream
+    st = lib.vpp_chunk_attn_host_fwd(ctypes.byref(hargs), ctypes.c_void_p(stream))
+    if st != 0:
+        raise VppError(st, "%s: %s" % (lib.vpp_status_string(st).decode(), lib.vpp_host_last_error().decode()))
+
+
 class HostChunkPipeline:
-    """One request's chunk whose inputs and outputs live in pinned host memory, streamed through the GPU in slices.
+    """Argument holder for vpp_chunk_attn_host_fwd: one request's chunk whose query, new K/V rows and results live in
+    pinned host memory.  All of the work (slicing, copies, append, attention) is the C entry point's; this class only
+    owns the device staging buffers and the argument struct."""
 
-    The chunk's query rows are cut into `slices` runs.  Slice i's query rows and the cache pages that hold its own keys
-    and values go host -> device on a copy stream; its attention (prefix = the request's prefix plus the earlier slices,
-    whose pages are in the cache by then) is enqueued on the compute stream as soon as they have landed; its output rows
-    go device -> host on a third stream.  Copies of one slice overlap the attention of its neighbours; every slice is one
-    vpp_chunk_attn_fwd call.  A step is self-contained: nothing of the next step starts before the last copy of this one."""
-
-    @staticmethod
-    def plan_slices(prefix, chunk, block_size, num_q_heads, num_kv_heads, sm_count):
-        """Three slices (first, middle, last) of whole 128-row tiles.  What a step cannot overlap is the first copy in, the
-        last copy out and, per launch, the idle part of its last wave of work items (an item is one query tile of one
-        pair of q-heads and runs for as long as the prefix is long): pick the lengths that make the sum smallest."""
-        step = max(128, block_size)
-        tiles = chunk // step
-        if chunk % step or tiles < 3:
-            return [chunk]
-        group = num_q_heads // num_kv_heads
-        items_per_tile = (step // 128) * (num_q_heads // 2 if group % 2 == 0 else num_q_heads)
-        item_ms = (prefix + chunk / 2) / 128 * 2.0e-3                 # ~2 us per KV tile of an item
-        in_ms, out_ms = 0.038 * step / 128, 0.030 * step / 128        # copy time per tile of rows (q in, out back) at ~55 GB/s
-
-        def idle(k):
-            w = k * items_per_tile / sm_count
-            return (-(-k * items_per_tile // sm_count) - w) * item_ms
-
-        best = None
-        for a in range(1, tiles - 1):
-            for c in range(1, tiles - a):
-                b = tiles - a - c
-                cost = a * in_ms + c * out_ms + idle(a) + idle(b) + idle(c)
-                if best is None or cost < best[0]:
-                    best = (cost, [a * step, b * step, c * step])
-        return best[1]
-
-    def __init__(self, prob, slices="auto", num_kv_splits=0):
-        """slices: "auto" (plan_slices), a count (equal slices) or a list of slice lengths in query rows (each a multiple of
-        the page size)."""
+    def __init__(self, prob, slices=None, num_kv_splits=0, want_lse=True):
+        """prob: a one-request Problem on the GPU (its cache holds the prefix; the chunk's own rows are written by the
+        call).  slices: None (the library plans) or a list of slice lengths in query rows."""
         assert prob.num_reqs == 1 and prob.block_table is not None
         dev = prob.q.device
-        P, C, B = int(prob.prefix_len[0]), int(prob.chunk_len[0]), prob.block_size
-        if slices == "auto":
-            slices = self.plan_slices(P, C, B, prob.num_q_heads, prob.num_kv_heads,
-                                      torch.cuda.get_device_properties(dev).multi_processor_count)
-        lens = [C // slices] * slices if isinstance(slices, int) else [int(x) for x in slices]
-        assert sum(lens) == C and all(n > 0 and n % B == 0 for n in lens) and P % B == 0, "slices must cover whole cache pages"
-        slices = len(lens)
-        bounds = [0]
-        for n in lens:
-            bounds.append(bounds[-1] + n)
-        self.prob, self.slices = prob, slices
+        P, C = int(prob.prefix_len[0]), int(prob.chunk_len[0])
+        self.prob, self.P, self.C = prob, P, C
+        aliased = prob.v_cache.data_ptr() == prob.k_cache.data_ptr()
+        self.q_dev = torch.empty_like(prob.q)
         self.out = torch.empty((C, prob.num_q_heads, prob.head_dim_v), dtype=torch.bfloat16, device=dev)
-        self.lse = torch.empty((C, prob.num_q_heads), dtype=torch.float32, device=dev)
-        self.status = torch.zeros(slices, dtype=torch.int32, device=dev)
-        self.parts = []
-        bt = prob.block_table[0].cpu().tolist()
-        for i in range(slices):
-            lo, hi = bounds[i], bounds[i + 1]
-            pre = torch.tensor([P + lo], dtype=torch.int32, device=dev)
-            cl = torch.tensor([hi - lo], dtype=torch.int32, device=dev)
-            a = make_args(prob.q[lo:hi], prob.k_cache, prob.v_cache, prob.block_table, pre, cl, B, prob.max_seq_len,
-                          prob.scale, num_kv_splits=num_kv_splits, out=self.out[lo:hi], lse=self.lse[lo:hi],
-                          status=self.status[i:i + 1], head_dim_v=prob.head_dim_v)
-            ws = torch.empty(max(vpp_chunk_attn_workspace_size(a), 256), dtype=torch.uint8, device=dev)
-            a.workspace, a.workspace_bytes = _ptr(ws), ws.numel()
-            blocks = [bt[j] for j in range((P + lo) // B, (P + hi) // B)]
-            self.parts.append((lo, hi, a, ws, pre, cl, blocks))
-        self.s_in, self.s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-        self.ev_in = [torch.cuda.Event() for _ in range(slices)]
-        self.ev_done = [torch.cuda.Event() for _ in range(slices)]
-        self.ev_start, self.ev_end = torch.cuda.Event(), torch.cuda.Event()
+        self.lse = torch.empty((C, prob.num_q_heads), dtype=torch.float32, device=dev) if want_lse else None
+        self.k_new_dev = torch.empty((C, prob.num_kv_heads, prob.head_dim_qk), dtype=torch.bfloat16, device=dev)
+        self.v_new_dev = None if aliased else torch.empty((C, prob.num_kv_heads, prob.head_dim_v), dtype=torch.bfloat16, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        h = HostChunkAttnArgs()
+        h.dev = make_args(self.q_dev, prob.k_cache, prob.v_cache, prob.block_table, prob.prefix_len, prob.chunk_len,
+                          prob.block_size, prob.max_seq_len, prob.scale, num_kv_splits=num_kv_splits, out=self.out,
+                          lse=self.lse, status=self.status, head_dim_v=prob.head_dim_v)
+        h.prefix_len, h.chunk_len = P, C
+        self._slice_rows = None
+        if slices is not None:
+            self._slice_rows = (ctypes.c_int32 * len(slices))(*[int(x) for x in slices])
+            h.slice_rows, h.num_slices = ctypes.cast(self._slice_rows, ctypes.c_void_p), len(slices)
+        h.k_new_dev = _ptr(self.k_new_dev)
+        h.v_new_dev = _ptr(self.v_new_dev) if self.v_new_dev is not None else None
+        self.hargs = h
+        n = vpp_chunk_attn_host_workspace_size(h)
+        if n == 0:
+            raise VppError(-1, load_library().vpp_host_last_error().decode())
+        self.workspace = torch.empty(n, dtype=torch.uint8, device=dev)
+        h.dev.workspace, h.dev.workspace_bytes = _ptr(self.workspace), n
+        self.slices = vpp_chunk_attn_host_plan(h)
 
-    def chunk_blocks(self):
-        """Physical cache blocks of the chunk's own positions, in order."""
-        return [b for part in self.parts for b in part[6]]
-
-    def run(self, q_host, k_pages_host, v_pages_host, out_host, lse_host, stream):
-        """q_host [C, Hq, Dqk], k_pages_host / v_pages_host: dicts block -> pinned page tensors, out_host / lse_host pinned.
-        `stream` (a torch.cuda.Stream) is the compute stream; on return it waits for the last device -> host copy."""
+    def chunk_rows(self, cache):
+        """The chunk's own rows of a [blocks, block_size, Hkv, D] cache tensor, token-major (what k_new / v_new hold)."""
         p = self.prob
-        self.ev_start.record(stream)
-        self.s_in.wait_event(self.ev_start)
-        self.s_out.wait_event(self.ev_start)
-        for i, (lo, hi, a, _ws, _pre, _cl, blocks) in enumerate(self.parts):
-            with torch.cuda.stream(self.s_in):
-                p.q[lo:hi].copy_(q_host[lo:hi], non_blocking=True)
-                for b in blocks:
-                    p.k_cache[b].copy_(k_pages_host[b], non_blocking=True)
-                    p.v_cache[b].copy_(v_pages_host[b], non_blocking=True)
-                self.ev_in[i].record(self.s_in)
-            stream.wait_event(self.ev_in[i])
-            vpp_chunk_attn_fwd(a, stream.cuda_stream)
-            self.ev_done[i].record(stream)
-            with torch.cuda.stream(self.s_out):
-                self.s_out.wait_event(self.ev_done[i])
-                out_host[lo:hi].copy_(self.out[lo:hi], non_blocking=True)
-                lse_host[lo:hi].copy_(self.lse[lo:hi], non_blocking=True)
-        self.ev_end.record(self.s_out)
-        stream.wait_event(self.ev_end)
+        pos = torch.arange(self.P, self.P + self.C, device=p.block_table.device)
+        blk = p.block_table[0, (pos // p.block_size).long()].long()
+        return cache[blk.to(cache.device), (pos % p.block_size).long().to(cache.device)]
+
+    def run(self, q_host, k_new_host, v_new_host, out_host, lse_host, stream=None):
+        """Host tensors (pinned for overlap): q [C, Hq, Dqk], k_new [C, Hkv, Dqk], v_new [C, Hkv, Dv] (None under MLA
+        aliasing), out [C, Hq, Dv], lse [C, Hq] or None.  Enqueues everything; `stream` ends up waiting for the last
+        device -> host copy."""
+        h = self.hargs
+        h.q_host, h.k_new_host = q_host.data_ptr(), k_new_host.data_ptr()
+        h.v_new_host = v_new_host.data_ptr() if v_new_host is not None else None
+        h.out_host = out_host.data_ptr()
+        h.lse_host = lse_host.data_ptr() if lse_host is not None else None
+        vpp_chunk_attn_host_fwd(h, stream)
+
+

@@ -7,7 +7,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvpp_chunk_attn.so")
-SOURCES = ["api.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "noalloc.cu", "host_pipeline.cu"]
 
 
 def _nvcc():

@@ -35,7 +35,7 @@ def compare(out_gpu, lse_gpu, prob_cpu, rows, label=""):
     ref_o, ref_l = oracle_rows(prob_cpu, rows)
     ti, hi = packed_index(prob_cpu, rows)
     got_o = out_gpu.float().cpu().numpy().astype(np.float64)[ti, hi]
-    got_l = lse_gpu.cpu().numpy().astype(np.float64)[ti, hi]
+    got_l = lse_gpu.cpu().numpy().astype(np.float64)[ti, hi] if lse_gpu is not None else ref_l   # (None: out only)
     assert np.isfinite(got_o).all(), "%s: non-finite output" % label
     err = np.abs(got_o - ref_o)
     allowed = np.maximum(ABS_TOL, 2.0 ** -8 * np.abs(ref_o))

@@ -109,6 +109,82 @@ int main(int argc, char** argv) {
 '''
 
 
+C_SOURCE_HOST = r'''
+#include <cuda_runtime_api.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include "vpp.h"
+
+#define CK(x) do { cudaError_t e_ = (x); if (e_ != cudaSuccess) { fprintf(stderr, "%s: %s\n", #x, cudaGetErrorString(e_)); return 2; } } while (0)
+
+/* one request's chunk from page-locked host memory through vpp_chunk_attn_host_fwd */
+int main(int argc, char** argv) {
+    if (argc != 3) return 1;
+    FILE* f = fopen(argv[1], "rb");
+    if (!f) return 1;
+    int32_t h[12];   /* P, C, Hq, Hkv, D, B, num_blocks, max_blocks, max_seq, splits */
+    if (fread(h, 4, 12, f) != 12) return 3;
+    const int P = h[0], C = h[1], Hq = h[2], Hkv = h[3], D = h[4], B = h[5], NB = h[6], MB = h[7], MAXSEQ = h[8], S = h[9];
+    float scale;
+    if (fread(&scale, 4, 1, f) != 1) return 3;
+    const size_t q_bytes = (size_t)C * Hq * D * 2, n_bytes = (size_t)C * Hkv * D * 2, c_bytes = (size_t)NB * B * Hkv * D * 2;
+    void *q, *kn, *vn, *out; float* lse;
+    CK(cudaMallocHost(&q, q_bytes)); CK(cudaMallocHost(&kn, n_bytes)); CK(cudaMallocHost(&vn, n_bytes));
+    CK(cudaMallocHost(&out, q_bytes)); CK(cudaMallocHost((void**)&lse, (size_t)C * Hq * 4));
+    void* cache = malloc(2 * c_bytes);
+    int32_t* bt = (int32_t*)malloc((size_t)MB * 4);
+    if (fread(q, 1, q_bytes, f) != q_bytes || fread(cache, 1, 2 * c_bytes, f) != 2 * c_bytes || fread(kn, 1, n_bytes, f) != n_bytes ||
+        fread(vn, 1, n_bytes, f) != n_bytes || fread(bt, 4, MB, f) != (size_t)MB) return 3;
+    fclose(f);
+    void *dq, *dk, *dv, *dkn, *dvn, *dbt, *dout, *dlse, *dst, *dws;
+    CK(cudaMalloc(&dq, q_bytes)); CK(cudaMalloc(&dk, c_bytes)); CK(cudaMalloc(&dv, c_bytes)); CK(cudaMalloc(&dkn, n_bytes));
+    CK(cudaMalloc(&dvn, n_bytes)); CK(cudaMalloc(&dbt, (size_t)MB * 4)); CK(cudaMalloc(&dout, q_bytes));
+    CK(cudaMalloc(&dlse, (size_t)C * Hq * 4)); CK(cudaMalloc(&dst, 4));
+    CK(cudaMemcpy(dk, cache, c_bytes, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(dv, (char*)cache + c_bytes, c_bytes, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(dbt, bt, (size_t)MB * 4, cudaMemcpyHostToDevice));
+    cudaStream_t stream;
+    CK(cudaStreamCreate(&stream));
+
+    vpp_chunk_attn_host_args a;
+    memset(&a, 0, sizeof a);
+    a.q_host = q; a.k_new_host = kn; a.v_new_host = vn; a.out_host = out; a.lse_host = lse;
+    a.prefix_len = P; a.chunk_len = C;
+    a.dev.q = dq; a.dev.k_cache = dk; a.dev.v_cache = dv;
+    a.dev.k_block_stride = a.dev.v_block_stride = (int64_t)B * Hkv * D;
+    a.dev.k_token_stride = a.dev.v_token_stride = (int64_t)Hkv * D;
+    a.dev.k_head_stride = a.dev.v_head_stride = D;
+    a.dev.block_table = (const int32_t*)dbt;
+    a.dev.num_reqs = 1; a.dev.max_blocks_per_req = MB; a.dev.block_size = B; a.dev.num_blocks = NB; a.dev.total_q = C;
+    a.dev.max_seq_len = MAXSEQ; a.dev.num_q_heads = Hq; a.dev.num_kv_heads = Hkv; a.dev.head_dim_qk = D; a.dev.head_dim_v = D;
+    a.dev.softmax_scale = scale; a.dev.num_kv_splits = S; a.dev.out = dout; a.dev.lse = (float*)dlse; a.dev.status = (int32_t*)dst;
+    a.k_new_dev = dkn; a.v_new_dev = dvn;
+    int32_t plan[VPP_HOST_MAX_SLICES];
+    const int n = vpp_chunk_attn_host_plan(&a, plan);
+    const size_t ws = vpp_chunk_attn_host_workspace_size(&a);
+    if (n == 0 || ws == 0) { fprintf(stderr, "plan: %s\n", vpp_host_last_error()); return 5; }
+    CK(cudaMalloc(&dws, ws));
+    a.dev.workspace = dws; a.dev.workspace_bytes = ws;
+    vpp_status st = vpp_chunk_attn_host_fwd(&a, stream);
+    if (st != VPP_OK) { fprintf(stderr, "%s: %s\n", vpp_status_string(st), vpp_host_last_error()); return 6; }
+    CK(cudaStreamSynchronize(stream));
+    int32_t status;
+    CK(cudaMemcpy(&status, dst, 4, cudaMemcpyDeviceToHost));
+    if (status) { fprintf(stderr, "device status %d\n", status); return 7; }
+    FILE* g = fopen(argv[2], "wb");
+    fwrite(out, 1, q_bytes, g);
+    fwrite(lse, 1, (size_t)C * Hq * 4, g);
+    fclose(g);
+    printf("slices %d:", n);
+    for (int i = 0; i < n; ++i) printf(" %d", plan[i]);
+    printf(" workspace %zu\n", ws);
+    return 0;
+}
+'''
+
+
 def _bits(t):
     return t.contiguous().view(torch.int16).numpy().tobytes()
 
@@ -160,3 +236,42 @@ def test_a_plain_c_program_appends_a_chunk_and_attends(tmp_path, splits):
     lse = torch.from_numpy(raw[n_out:].view(np.float32).copy()).view(T, 8)
     rows = oracle.all_rows(prob.chunk_len.numpy(), 8)
     print(compare(out, lse, prob, rows, "C client S=%d" % splits), res.stdout.strip())
+
+
+def test_a_plain_c_program_runs_a_chunk_from_host_memory(tmp_path):
+    """The host entry point from plain C: page-locked buffers from cudaMallocHost, one call, results back in host memory."""
+    gcc = shutil.which("gcc")
+    cuda = "/usr/local/cuda"
+    if gcc is None or not os.path.exists(os.path.join(cuda, "include", "cuda_runtime_api.h")):
+        pytest.skip("no C toolchain / CUDA headers on this box")
+    api.load_library()
+    P, C = 384, 640
+    prob = W.make_problem(7200, [P], [C], 8, 2, 128, 128, block_size=64)
+    pos = torch.arange(P, P + C)
+    blk, slot = prob.block_table[0, (pos // 64).long()].long(), (pos % 64).long()
+    k_new, v_new = prob.k_cache[blk, slot].contiguous(), prob.v_cache[blk, slot].contiguous()
+    kc, vc = prob.k_cache.clone(), prob.v_cache.clone()
+    kc[blk, slot] = float("nan")
+    vc[blk, slot] = float("nan")
+    src, exe, fin, fout = tmp_path / "host_client.c", tmp_path / "host_client", tmp_path / "in.bin", tmp_path / "out.bin"
+    src.write_text(C_SOURCE_HOST)
+    lib_dir = os.path.dirname(api.LIB_PATH)
+    subprocess.check_call([gcc, "-O1", "-std=c11", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(cuda, "include"),
+                           "-o", str(exe), str(src), "-L", lib_dir, "-l:libvpp_chunk_attn.so", "-L", os.path.join(cuda, "lib64"),
+                           "-lcudart", "-Wl,-rpath," + lib_dir, "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+    head = np.array([P, C, 8, 2, 128, 64, kc.shape[0], prob.block_table.shape[1], prob.max_seq_len, 0, 0, 0], np.int32)
+    with open(fin, "wb") as f:
+        f.write(head.tobytes())
+        f.write(np.float32(prob.scale).tobytes())
+        for t in (prob.q, kc, vc, k_new, v_new):
+            f.write(_bits(t))
+        f.write(prob.block_table[0].numpy().astype(np.int32).tobytes())
+    res = subprocess.run([str(exe), str(fin), str(fout)], capture_output=True, text=True, timeout=120)
+    assert res.returncode == 0, res.stderr + res.stdout
+    assert "slices 3: 128 384 128" in res.stdout or "slices 3:" in res.stdout
+    raw = np.fromfile(fout, dtype=np.uint8)
+    n_out = C * 8 * 128 * 2
+    out = torch.from_numpy(raw[:n_out].view(np.int16).copy()).view(torch.bfloat16).view(C, 8, 128)
+    lse = torch.from_numpy(raw[n_out:].view(np.float32).copy()).view(C, 8)
+    rows = oracle.all_rows(prob.chunk_len.numpy(), 8)
+    print(compare(out, lse, prob, rows, "C host client"), res.stdout.strip())

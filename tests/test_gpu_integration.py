@@ -68,31 +68,85 @@ def test_one_chunk_step_replays_from_a_cuda_graph(splits):
     assert not torch.equal(runner2_out.view(torch.int16), eager.view(torch.int16))
 
 
-def test_host_streaming_pipeline_matches_the_oracle():
-    """A chunk streamed from pinned host memory in four slices (copies overlapping attention) gives the oracle's rows."""
+def _host_side(prob_cpu, prob, pipe):
+    """Pinned host copies of what vpp_chunk_attn_host_fwd brings in (q and the chunk's own K/V rows, token-major), with
+    those rows poisoned on the device beforehand, and pinned result buffers."""
+    aliased = prob_cpu.v_cache.data_ptr() == prob_cpu.k_cache.data_ptr()
+    q_host = prob_cpu.q.clone().pin_memory()
+    k_new = pipe.chunk_rows(prob_cpu.k_cache).contiguous().pin_memory()
+    v_new = None if aliased else pipe.chunk_rows(prob_cpu.v_cache).contiguous().pin_memory()
+    pos = torch.arange(pipe.P, pipe.P + pipe.C)
+    blk = prob_cpu.block_table[0, (pos // prob_cpu.block_size).long()].long().cuda()
+    slot = (pos % prob_cpu.block_size).long().cuda()
+    prob.k_cache[blk, slot] = float("nan")
+    if not aliased:
+        prob.v_cache[blk, slot] = float("nan")
+    C = pipe.C
+    out_host = torch.full((C, prob_cpu.num_q_heads, prob_cpu.head_dim_v), float("nan"), dtype=torch.bfloat16).pin_memory()
+    lse_host = torch.full((C, prob_cpu.num_q_heads), float("nan"), dtype=torch.float32).pin_memory()
+    return q_host, k_new, v_new, out_host, lse_host
+
+
+def test_host_entry_point_matches_the_oracle():
+    """vpp_chunk_attn_host_fwd: a chunk streamed from pinned host memory in four given slices (copies overlapping
+    append + attention) gives the oracle's rows, and the chunk's K/V rows end up in the cache bit for bit."""
     prob_cpu = W.make_problem(4300, [256], [512], 8, 2, 128, 128, block_size=64, std=0.7)
     prob = prob_cpu.to("cuda")
-    pipe = api.HostChunkPipeline(prob, slices=4)
-    q_host = prob_cpu.q.clone().pin_memory()
-    blocks = pipe.chunk_blocks()
-    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
-    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
-    # what the pipeline has to bring in is not on the device beforehand
-    prob.q.fill_(float("nan"))
-    for b in blocks:
-        prob.k_cache[b] = float("nan")
-        prob.v_cache[b] = float("nan")
-    out_host = torch.empty((512, 8, 128), dtype=torch.bfloat16).pin_memory()
-    lse_host = torch.empty((512, 8), dtype=torch.float32).pin_memory()
+    pipe = api.HostChunkPipeline(prob, slices=[128, 64, 192, 128])
+    assert pipe.slices == [128, 64, 192, 128]
+    q_host, k_new, v_new, out_host, lse_host = _host_side(prob_cpu, prob, pipe)
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
-    for _ in range(2):                       # a second step reuses every buffer and event
+    for _ in range(2):                       # a second step reuses every buffer, stream and event
         out_host.fill_(float("nan"))
-        pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+        pipe.run(q_host, k_new, v_new, out_host, lse_host, stream)
         stream.synchronize()
-        assert int(pipe.status.max().item()) == 0
+        assert int(pipe.status.item()) == 0
         rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
-        print(compare(out_host, lse_host, prob_cpu, rows, "host pipeline"))
+        print(compare(out_host, lse_host, prob_cpu, rows, "host entry point"))
+    live = torch.zeros(prob_cpu.k_cache.shape[:2], dtype=torch.bool)
+    for pos in range(256 + 512):
+        live[int(prob_cpu.block_table[0, pos // 64]), pos % 64] = True
+    assert torch.equal(prob.k_cache.cpu()[live].view(torch.int16), prob_cpu.k_cache[live].view(torch.int16))
+    assert torch.equal(prob.v_cache.cpu()[live].view(torch.int16), prob_cpu.v_cache[live].view(torch.int16))
+
+
+@pytest.mark.parametrize("case", ["mla", "ragged", "no_lse", "unaligned_prefix"])
+def test_host_entry_point_variants(case):
+    """The latent (MLA) cache whose values alias the keys, a ragged chunk (one slice), a call without lse, and a prefix
+    that is not a multiple of the page size (the rows are appended by the kernel, not copied page-wise)."""
+    if case == "mla":
+        prob_cpu = W.make_problem(4310, [320], [384], 16, 1, 576, 512, block_size=64, std=0.5, v_aliases_k=True)
+    elif case == "ragged":
+        prob_cpu = W.make_problem(4311, [100], [333], 8, 2, 128, 128, block_size=32, std=0.7)
+    elif case == "unaligned_prefix":
+        prob_cpu = W.make_problem(4313, [77], [512], 6, 2, 128, 128, block_size=16, std=0.7)
+    else:
+        prob_cpu = W.make_problem(4312, [128], [384], 4, 4, 128, 128, block_size=128, std=0.7)
+    prob = prob_cpu.to("cuda")
+    pipe = api.HostChunkPipeline(prob, want_lse=(case != "no_lse"))
+    assert sum(pipe.slices) == int(prob_cpu.chunk_len[0]) and len(pipe.slices) == (1 if case == "ragged" else 3)
+    q_host, k_new, v_new, out_host, lse_host = _host_side(prob_cpu, prob, pipe)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    pipe.run(q_host, k_new, v_new, out_host, None if case == "no_lse" else lse_host, stream)
+    stream.synchronize()
+    assert int(pipe.status.item()) == 0
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(case, pipe.slices, compare(out_host, None if case == "no_lse" else lse_host, prob_cpu, rows, "host entry point, " + case))
+
+
+def test_host_entry_point_refuses_bad_arguments():
+    prob = W.make_problem(4320, [256], [512], 8, 2, 128, 128, block_size=64).to("cuda")
+    with pytest.raises(api.VppError):
+        api.HostChunkPipeline(prob, slices=[128, 128])              # does not add up to the chunk
+    pipe = api.HostChunkPipeline(prob)
+    pipe.hargs.dev.workspace_bytes = 1024
+    q = torch.zeros((512, 8, 128), dtype=torch.bfloat16).pin_memory()
+    kv = torch.zeros((512, 2, 128), dtype=torch.bfloat16).pin_memory()
+    with pytest.raises(api.VppError) as e:
+        pipe.run(q, kv, kv, q.clone().pin_memory(), None)
+    assert e.value.status == api.VPP_ERR_WORKSPACE
 
 
 def test_sparse_attention_after_append_and_from_a_cuda_graph():
@@ -139,51 +193,20 @@ def test_sparse_attention_after_append_and_from_a_cuda_graph():
     assert (np.abs(got_l - ref_l)[both] <= 1e-5 * np.maximum(1.0, np.abs(ref_l[both]))).all()
 
 
-def test_host_streaming_pipeline_with_planned_slices():
-    """The default slice plan (first / middle / last slice of whole tiles) on a chunk of eight query tiles."""
-    prob_cpu = W.make_problem(4500, [512], [1024], 8, 2, 128, 128, block_size=128, std=0.7)
-    prob = prob_cpu.to("cuda")
-    pipe = api.HostChunkPipeline(prob)                      # slices="auto"
-    plan = [hi - lo for (lo, hi, *_r) in pipe.parts]
-    assert sum(plan) == 1024 and len(plan) == 3 and all(n % 128 == 0 and n > 0 for n in plan)
-    q_host = prob_cpu.q.clone().pin_memory()
-    blocks = pipe.chunk_blocks()
-    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
-    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
-    prob.q.fill_(float("nan"))
-    out_host = torch.empty((1024, 8, 128), dtype=torch.bfloat16).pin_memory()
-    lse_host = torch.empty((1024, 8), dtype=torch.float32).pin_memory()
-    stream = torch.cuda.Stream()
-    stream.wait_stream(torch.cuda.current_stream())
-    pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
-    stream.synchronize()
-    assert int(pipe.status.max().item()) == 0
-    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
-    print(plan, compare(out_host, lse_host, prob_cpu, rows, "planned slices"))
-
-
-def test_host_streaming_pipeline_at_benchmark_size_matches_the_oracle():
+def test_host_entry_point_at_benchmark_size_matches_the_oracle():
     """The end-to-end leg of bench.py at its real size: the cfg 2 chunk at prefix 65536 streamed from pinned host memory in
     the planned slices, compared with the oracle on one row of every (query tile, pair of q-heads) plus the edge rows."""
     from parity import sample_rows, tile_rows
     prob = W.cfg2(prefix=65536, device="cuda")
     prob_cpu = prob.to("cpu")
     pipe = api.HostChunkPipeline(prob)
-    q_host = prob_cpu.q.clone().pin_memory()
-    blocks = pipe.chunk_blocks()
-    k_pages = {b: prob_cpu.k_cache[b].clone().pin_memory() for b in blocks}
-    v_pages = {b: prob_cpu.v_cache[b].clone().pin_memory() for b in blocks}
-    prob.q.fill_(float("nan"))                      # what the pipeline brings in is not on the device beforehand
-    for b in blocks:
-        prob.k_cache[b] = float("nan")
-        prob.v_cache[b] = float("nan")
-    out_host = torch.full((8192, 64, 128), float("nan"), dtype=torch.bfloat16).pin_memory()
-    lse_host = torch.full((8192, 64), float("nan"), dtype=torch.float32).pin_memory()
+    assert pipe.slices == [1152, 5888, 1152]
+    q_host, k_new, v_new, out_host, lse_host = _host_side(prob_cpu, prob, pipe)
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
-    pipe.run(q_host, k_pages, v_pages, out_host, lse_host, stream)
+    pipe.run(q_host, k_new, v_new, out_host, lse_host, stream)
     stream.synchronize()
-    assert int(pipe.status.max().item()) == 0
+    assert int(pipe.status.item()) == 0
     assert torch.isfinite(out_host.float()).all() and torch.isfinite(lse_host).all()
     rows = np.unique(np.concatenate([sample_rows(prob_cpu, n_random=64), tile_rows(prob_cpu, per="pair", seed=3)]), axis=0)
-    print(compare(out_host, lse_host, prob_cpu, rows, "host pipeline, cfg2 at 65536"))
+    print(compare(out_host, lse_host, prob_cpu, rows, "host entry point, cfg2 at 65536"))

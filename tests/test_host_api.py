@@ -157,13 +157,57 @@ def test_flop_count_is_the_exact_causal_count():
     assert p.pairs() == pairs and p.flops() == 2 * 4 * (16 + 8) * pairs
 
 
-def test_pipeline_slice_plan_covers_the_chunk_in_whole_pages():
-    from paper_2608_26523_b200 import api
-    for prefix, chunk, bs, hq, hkv in [(65536, 8192, 128, 64, 4), (0, 8192, 128, 64, 8), (256, 512, 64, 8, 2), (4096, 1024, 256, 16, 16)]:
-        plan = api.HostChunkPipeline.plan_slices(prefix, chunk, bs, hq, hkv, 148)
-        assert sum(plan) == chunk and all(n > 0 and n % bs == 0 for n in plan)
+def _host_plan_args(prefix, chunk, hq, hkv, dqk=128, dv=128, slices=None):
+    h = api.HostChunkAttnArgs()
+    h.dev.num_reqs, h.dev.total_q, h.dev.max_seq_len = 1, chunk, prefix + chunk
+    h.dev.num_q_heads, h.dev.num_kv_heads, h.dev.head_dim_qk, h.dev.head_dim_v = hq, hkv, dqk, dv
+    h.prefix_len, h.chunk_len = prefix, chunk
+    if slices is not None:
+        keep = (ctypes.c_int32 * len(slices))(*slices)
+        h.slice_rows, h.num_slices = ctypes.cast(keep, ctypes.c_void_p), len(slices)
+        h._keep = keep
+    return h
+
+
+def test_host_entry_point_slice_plan():
+    """The planner of vpp_chunk_attn_host_fwd is host arithmetic: whole 128-row tiles that cover the chunk; ragged or
+    short chunks in one slice; given slices are checked."""
+    for prefix, chunk, hq, hkv in [(65536, 8192, 64, 4), (0, 8192, 64, 8), (256, 512, 8, 2), (4096, 1024, 16, 16)]:
+        plan = api.vpp_chunk_attn_host_plan(_host_plan_args(prefix, chunk, hq, hkv))
+        assert len(plan) == 3 and sum(plan) == chunk and all(n > 0 and n % 128 == 0 for n in plan)
     # the benchmark's chunk: first and last slice close to two full waves of work items, the middle one to ten
-    assert api.HostChunkPipeline.plan_slices(65536, 8192, 128, 64, 4, 148) == [1152, 5888, 1152]
+    assert api.vpp_chunk_attn_host_plan(_host_plan_args(65536, 8192, 64, 4)) == [1152, 5888, 1152]
+    assert api.vpp_chunk_attn_host_plan(_host_plan_args(100, 333, 8, 2)) == [333]
+    assert api.vpp_chunk_attn_host_plan(_host_plan_args(0, 256, 8, 2)) == [256]
+    assert api.vpp_chunk_attn_host_plan(_host_plan_args(0, 512, 8, 2, slices=[100, 412])) == [100, 412]
+    lib = api.load_library()
+    for bad in [_host_plan_args(0, 512, 8, 2, slices=[100, 400]), _host_plan_args(0, 512, 8, 2, slices=[600, -88]),
+                _host_plan_args(0, 512, 8, 3), _host_plan_args(0, 512, 8, 2, slices=[32] * 16 + [0])]:
+        assert api.vpp_chunk_attn_host_plan(bad) == [] and lib.vpp_host_last_error() != b""
+    bad = _host_plan_args(0, 512, 8, 2)
+    bad.dev.num_reqs = 2
+    assert api.vpp_chunk_attn_host_plan(bad) == [] and api.vpp_chunk_attn_host_workspace_size(bad) == 0
+    bad = _host_plan_args(10, 512, 8, 2)
+    bad.dev.max_seq_len = 500
+    assert api.vpp_chunk_attn_host_plan(bad) == []
+
+
+def test_host_entry_point_workspace_is_the_sum_of_its_slices():
+    h = _host_plan_args(65536, 8192, 64, 4)
+    h.dev.block_size, h.dev.max_blocks_per_req, h.dev.num_blocks = 128, 640, 640
+    h.dev.k_block_stride = h.dev.v_block_stride = 128 * 4 * 128
+    h.dev.k_token_stride = h.dev.v_token_stride = 4 * 128
+    h.dev.k_head_stride = h.dev.v_head_stride = 128
+    h.dev.softmax_scale = 0.088
+    fake = ctypes.c_void_p(1 << 20)
+    h.dev.q = h.dev.k_cache = h.dev.v_cache = h.dev.block_table = h.dev.prefix_len = h.dev.chunk_len = h.dev.out = fake
+    total = api.vpp_chunk_attn_host_workspace_size(h)
+    parts = 0
+    for rows in (1152, 5888, 1152):
+        a = api.ChunkAttnArgs.from_buffer_copy(h.dev)
+        a.total_q = rows
+        parts += (api.vpp_chunk_attn_workspace_size(a) + 255) // 256 * 256
+    assert total == 256 + parts
 
 
 def _fake_args(total_q, num_reqs, hq, hkv, max_seq_len, num_kv_splits):
