@@ -44,6 +44,8 @@ constexpr float kRescaleThreshold = 8.f;      // log2 units
 // 0: P is handed to the MMA thread whole; c in 1..3: the first 32*c key columns are handed over early so that
 // O += P V can start on them while the rest of the exponentials are computed
 constexpr int kSplitChunks = 1;
+constexpr int kPartWaitDefer = 8;             // pairs of columns of the next chunk computed before that hand-over's store is awaited (0: none)
+static_assert(kPartWaitDefer >= 0 && kPartWaitDefer <= 16 && (kSplitChunks < 4 || kPartWaitDefer == 0), "the deferred wait needs a next chunk");
 
 struct WsItem {
     WorkUnit u;
@@ -630,6 +632,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
                 const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
                 float sum0 = 0.f, sum1 = 0.f;
+                // The wait for the early hand-over's store comes kPartWaitDefer pairs into the next chunk, so that the warp keeps
+                // issuing exponentials while the store completes.
+                constexpr int kDefer = kPartWaitDefer;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t pk[16];
@@ -641,9 +646,15 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
+                        if (kSplitChunks > 0 && c == kSplitChunks && (i >> 1) == kDefer - 1) {
+                            tc_wait_st();
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_p_part + 8 * t);
+                        }
                     }
                     tmem_st16(tS + c * 16, pk);
-                    if (kSplitChunks > 0 && c == kSplitChunks - 1) {
+                    if (kSplitChunks > 0 && c == kSplitChunks - 1 && kDefer == 0) {
                         tc_wait_st();
                         tc_fence_before();
                         __syncwarp();
