@@ -43,9 +43,12 @@ constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*al
 constexpr float kRescaleThreshold = 8.f;      // log2 units
 // 0: P is handed to the MMA thread whole; c in 1..3: the first 32*c key columns are handed over early so that
 // O += P V can start on them while the rest of the exponentials are computed
-constexpr int kSplitChunks = 1;
+// Early hand-overs of P: bit c set = the key columns up to 32 (c + 1) are handed to the MMA thread as soon as they are in
+// tensor memory, so that O += P V starts on them while the rest of the exponentials are computed (0: P is handed over whole).
+constexpr int kPartMask = 3;   // after 32 and after 64 columns (measured best: a hand-over after 96 columns costs more than it gains)
+static_assert(kPartMask >= 0 && kPartMask < 8, "hand-overs after 32, 64 and 96 columns only");
 constexpr int kPartWaitDefer = 8;             // pairs of columns of the next chunk computed before that hand-over's store is awaited (0: none)
-static_assert(kPartWaitDefer >= 0 && kPartWaitDefer <= 16 && (kSplitChunks < 4 || kPartWaitDefer == 0), "the deferred wait needs a next chunk");
+static_assert(kPartWaitDefer >= 1 && kPartWaitDefer <= 16, "the wait sits inside the next chunk");
 
 struct WsItem {
     WorkUnit u;
@@ -147,7 +150,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // Two slots used alternately: the producer can fix up the V tile of the next short item before the MMA thread has
     // looked at the barrier for this one (slot k & 1 for the k-th such tile, 24 bytes apart).
     const uint32_t bar_vfix = sBar + 96;
-    const uint32_t bar_p_part = sBar + 104;      // [2] first kSplitCols key columns of P are in place (optional early hand-off)
+    // [3][2] early hand-overs of P: part c (the key columns up to 32 (c + 1)) of tile t is in place.  One barrier per part:
+    // the MMA thread may look at part 0 only after part 1 has arrived too, which a shared barrier could not tell apart.
+    const uint32_t bar_p_part = sBar + 208;
     const uint32_t bar_kv_full = sBar + 128;     // [kWsStages]
     const uint32_t bar_kv_empty = sBar + 128 + 8 * kWsStages;
     const uint32_t bar_x1 = sBar + 128 + 16 * kWsStages;       // packed item: group 1 has published its (m, l) per row
@@ -168,7 +173,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(bar_item_empty + 8 * i, 9);
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_p_full + 8 * i, 4);   // one arrival per softmax warp
-            mbar_init(bar_p_part + 8 * i, 4);
+            for (int c = 0; c < 3; ++c) mbar_init(bar_p_part + 16 * c + 8 * i, 4);
             mbar_init(bar_o_full + 8 * i, 1);
         }
         mbar_init(bar_q_full, 1);
@@ -379,6 +384,24 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     mma_ts_lh(tO, tP + k * 8, v_lo + k * (2048 >> 4), kHi, kIdescPV, (!first || k > 0) ? 1u : 0u);
                 }
             };
+            // O_t += P_t V for one KV tile, following the hand-overs: every early part as soon as it is there, the rest after
+            // the whole of P.  pit = hand-overs of P_t seen so far (tile visits).
+            auto pv_tile = [&](int t, uint32_t tO, uint32_t tS, uint32_t v_stage, bool first, uint32_t pit, int where) -> bool {
+                int k0 = 0;
+#pragma unroll
+                for (int c = 0; c < 3; ++c) {
+                    if ((kPartMask >> c) & 1) {
+                        if (!wait1(bar_p_part + 16 * c + 8 * t, pit & 1, where)) return false;
+                        tc_fence_after();
+                        issue_pv(tO, tS, v_stage, first, k0, 2 * (c + 1));
+                        k0 = 2 * (c + 1);
+                    }
+                }
+                if (!wait1(bar_p_full + 8 * t, pit & 1, where + 1)) return false;
+                tc_fence_after();
+                issue_pv(tO, tS, v_stage, first, k0, 8);
+                return true;
+            };
             while (true) {
                 const uint32_t slot = item_it & 1;
                 if (!wait1(bar_item_full + 8 * slot, (item_it >> 1) & 1, 301)) break;
@@ -423,16 +446,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                             ++vfix_it;
                         }
                         const uint32_t tO = t ? tO1 : tO0, tS = t ? tS1 : tS0;
-                        if (kSplitChunks > 0) {
-                            ok = wait1(bar_p_part + 8 * t, pit & 1, 324);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_pv(tO, tS, sKV + st * kTileBytes, jj < 2, 0, 2 * kSplitChunks);
-                        }
-                        ok = wait1(bar_p_full + 8 * t, pit & 1, 325);
+                        ok = pv_tile(t, tO, tS, sKV + st * kTileBytes, jj < 2, pit, 324);
                         if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(tO, tS, sKV + st * kTileBytes, jj < 2, kSplitChunks > 0 ? 2 * kSplitChunks : 0, 8);
                         tc_commit(bar_kv_empty + 8 * st);
                         if (t) ++p_it1; else ++p_it;
                         if (jj + 2 < n) ok = do_qk(jj + 2);
@@ -470,23 +485,8 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     const bool has_next = jj + 1 < n;
                     stK = kv_it % kWsStages;
                     // ---- tile 0 ----
-                    if (kSplitChunks == 0) {
-                        ok = wait1(bar_p_full, p_it & 1, 306);
-                        if (!ok) break;
-                        tc_fence_after();
-                    }
-                    if (kSplitChunks > 0) {
-                        ok = wait1(bar_p_part, p_it & 1, 311);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 2 * kSplitChunks);
-                        ok = wait1(bar_p_full, p_it & 1, 306);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 2 * kSplitChunks, 8);
-                    } else {
-                        issue_pv(tO0, tS0, sKV + stV * kTileBytes, jj == 0, 0, 8);
-                    }
+                    ok = pv_tile(0, tO0, tS0, sKV + stV * kTileBytes, jj == 0, p_it, 308);
+                    if (!ok) break;
                     if (has_next) {
                         ok = wait1(bar_kv_full + 8 * stK, (kv_it / kWsStages) & 1, 307);
                         if (!ok) break;
@@ -499,17 +499,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         tc_commit(bar_o_full);
                     }
                     // ---- tile 1 ----
-                    if (kSplitChunks > 0) {
-                        ok = wait1(bar_p_part + 8, p_it1 & 1, 312);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, 0, 2 * kSplitChunks);
-                    }
-                    ok = wait1(bar_p_full + 8, p_it1 & 1, 308);
+                    ok = pv_tile(1, tO1, tS1, sKV + stV * kTileBytes, jj == 0, p_it1, 312);
                     if (!ok) break;
-                    tc_fence_after();
                     if (lane == 0) {
-                        issue_pv(tO1, tS1, sKV + stV * kTileBytes, jj == 0, kSplitChunks > 0 ? 2 * kSplitChunks : 0, 8);
                         tc_commit(bar_kv_empty + 8 * stV);
                         if (has_next) {
                             issue_qk(tS1, q_lo1, sKV + stK * kTileBytes);
@@ -576,7 +568,9 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) {
-                        if (kSplitChunks > 0) mbar_arrive(bar_p_part + 8 * t);
+#pragma unroll
+                        for (int c = 0; c < 3; ++c)
+                            if ((kPartMask >> c) & 1) mbar_arrive(bar_p_part + 16 * c + 8 * t);
                         mbar_arrive(bar_p);
                     }
                     continue;
@@ -646,20 +640,14 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         sum0 += p0;
                         sum1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
-                        if (kSplitChunks > 0 && c == kSplitChunks && (i >> 1) == kDefer - 1) {
+                        if (c > 0 && ((kPartMask >> (c - 1)) & 1) && (i >> 1) == kDefer - 1) {
                             tc_wait_st();
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_p_part + 8 * t);
+                            if (lane == 0) mbar_arrive(bar_p_part + 16 * (c - 1) + 8 * t);
                         }
                     }
                     tmem_st16(tS + c * 16, pk);
-                    if (kSplitChunks > 0 && c == kSplitChunks - 1 && kDefer == 0) {
-                        tc_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_p_part + 8 * t);
-                    }
                 }
                 l_run += sum0 + sum1;
                 tc_wait_st();
