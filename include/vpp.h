@@ -294,6 +294,7 @@ vpp_status vpp_kv_append(const vpp_kv_append_args *args, vpp_stream_t stream);
  *              (v_new_dev may be NULL under MLA aliasing).
  * Calls on one device are enqueued one at a time (a process-wide lock) and share two copy streams and their events,
  * created on the first call on that device (not a stream operation: make that first call outside any capture).
+ * After that the call can be captured in a CUDA graph like any fork-join of streams; a replay reads the host buffers anew.
  * On return everything is enqueued and `stream` waits for the last device -> host copy.  Errors: as
  * vpp_chunk_attn_fwd and vpp_kv_append (vpp_host_last_error() has the detail); VPP_ERR_CUDA if a copy or an event
  * operation fails -- earlier slices may have been enqueued by then.

@@ -136,6 +136,39 @@ def test_host_entry_point_variants(case):
     print(case, pipe.slices, compare(out_host, None if case == "no_lse" else lse_host, prob_cpu, rows, "host entry point, " + case))
 
 
+def test_host_entry_point_in_a_cuda_graph():
+    """The whole chunk step from host memory (copies in, append, attention, copies out, three streams) captured once in a
+    CUDA graph and replayed with new contents in the same pinned buffers."""
+    prob_cpu = W.make_problem(4330, [256], [512], 8, 2, 128, 128, block_size=64, std=0.7)
+    prob = prob_cpu.to("cuda")
+    pipe = api.HostChunkPipeline(prob)
+    q_host, k_new, v_new, out_host, lse_host = _host_side(prob_cpu, prob, pipe)
+    warm = torch.cuda.Stream()
+    warm.wait_stream(torch.cuda.current_stream())
+    pipe.run(q_host, k_new, v_new, out_host, lse_host, warm)       # first call on the device: creates the copy streams
+    warm.synchronize()
+    eager = out_host.clone()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        side.wait_stream(torch.cuda.current_stream())
+        graph.capture_begin()
+        pipe.run(q_host, k_new, v_new, out_host, lse_host, side)
+        graph.capture_end()
+    out_host.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out_host.view(torch.int16), eager.view(torch.int16))
+    # new queries in the same pinned buffer: the replay reads them
+    q_host.mul_(-1.0)
+    graph.replay()
+    torch.cuda.synchronize()
+    flipped = prob_cpu.to("cpu")
+    flipped.q = -prob_cpu.q
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(compare(out_host, lse_host, flipped, rows, "host entry point, graph replay"))
+
+
 def test_host_entry_point_refuses_bad_arguments():
     prob = W.make_problem(4320, [256], [512], 8, 2, 128, 128, block_size=64).to("cuda")
     with pytest.raises(api.VppError):
