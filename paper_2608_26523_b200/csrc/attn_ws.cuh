@@ -39,6 +39,9 @@ constexpr int kWsRegsLow = 72, kWsRegsHigh = 216;
 static_assert(kWsRegsLow + 2 * kWsRegsHigh <= 3 * 168 && kWsRegsLow % 8 == 0 && kWsRegsHigh % 8 == 0, "register budget");
 constexpr int kWsStages = 4;                  // 32 KB each
 constexpr int kTileBytes = 2 * kSlabBytes;    // one 128 x 128 bf16 tile
+// (the two alternating slots of the V-tail barrier cover a producer that runs at most two V tiles ahead of the MMA thread:
+//  a ring of more than four stages would need more slots -- five stages failed parity on short items)
+static_assert(kWsStages <= 4, "V-tail barrier slots");
 constexpr int kWsSmemBytes = 2 * kTileBytes + kWsStages * kTileBytes + 1024 /*align*/ + 2048 /*barriers, ring, merge exchange*/;
 constexpr float kRescaleThreshold = 8.f;      // log2 units
 // 0: P is handed to the MMA thread whole; c in 1..3: the first 32*c key columns are handed over early so that
