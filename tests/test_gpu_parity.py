@@ -195,3 +195,34 @@ def test_many_short_requests_with_ragged_single_tiles():
     out, lse, _ = run_gpu(prob_cpu.to("cuda"))
     rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
     print(compare(out, lse, prob_cpu, rows, "short ragged items"))
+
+
+@pytest.mark.parametrize("layout", ["head_major", "padded_rows", "k_and_v_interleaved"])
+@pytest.mark.parametrize("block_size", [128, 32])
+def test_cache_layouts_given_by_strides(layout, block_size):
+    """The caches are described by strides, not by a fixed layout: pages stored head-major ([block][kv-head][slot][d]), rows
+    padded to a larger token stride, and K and V interleaved in one allocation all give the same rows as the oracle (which
+    reads the logical tensors)."""
+    prob_cpu = W.make_problem(9300 + block_size, [300, 0, 77], [260, 200, 3], 8, 2, 128, 128, block_size=block_size, std=0.8)
+    prob = prob_cpu.to("cuda")
+    k, v = prob.k_cache, prob.v_cache                      # logical [blocks, slots, kv-heads, d]
+    nb, bs, hk, d = k.shape
+    if layout == "head_major":
+        k2 = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+        v2 = v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    elif layout == "padded_rows":
+        store_k = torch.full((nb, bs, hk + 1, d), float("nan"), dtype=k.dtype, device=k.device)
+        store_v = torch.full((nb, bs, hk + 1, d), float("nan"), dtype=k.dtype, device=k.device)
+        store_k[:, :, :hk] = k
+        store_v[:, :, :hk] = v
+        k2, v2 = store_k[:, :, :hk], store_v[:, :, :hk]
+    else:
+        store = torch.empty((nb, bs, hk, 2, d), dtype=k.dtype, device=k.device)
+        store[:, :, :, 0] = k
+        store[:, :, :, 1] = v
+        k2, v2 = store[:, :, :, 0], store[:, :, :, 1]
+    assert torch.equal(k2.view(torch.int16), k.view(torch.int16)) and k2.stride() != k.stride()
+    prob.k_cache, prob.v_cache = k2, v2
+    out, lse, _ = run_gpu(prob, 0)
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(layout, compare(out, lse, prob_cpu, rows, "layout " + layout))
