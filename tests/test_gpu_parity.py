@@ -226,3 +226,21 @@ def test_cache_layouts_given_by_strides(layout, block_size):
     out, lse, _ = run_gpu(prob, 0)
     rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
     print(layout, compare(out, lse, prob_cpu, rows, "layout " + layout))
+
+
+@pytest.mark.parametrize("block_size", [64, 16])
+def test_mla_latent_rows_with_a_padded_stride(block_size):
+    """The absorbed-MLA cache with its 576-feature rows 640 elements apart (values still alias the first 512 features of
+    the keys): both MLA kernels (pages of 64 tokens and smaller ones) read through the strides."""
+    prob_cpu = W.make_problem(9400 + block_size, [333, 0], [200, 140], 16, 1, 576, 512, block_size=block_size, std=0.5,
+                              v_aliases_k=True)
+    prob = prob_cpu.to("cuda")
+    nb, bs, hk, d = prob.k_cache.shape
+    store = torch.full((nb, bs, hk, 640), float("nan"), dtype=torch.bfloat16, device="cuda")
+    store[..., :576] = prob.k_cache
+    prob.k_cache = store[..., :576]
+    prob.v_cache = store[..., :512]
+    assert prob.k_cache.stride(1) == 640 and prob.v_cache.data_ptr() == prob.k_cache.data_ptr()
+    out, lse, _ = run_gpu(prob, 0)
+    rows = oracle.all_rows(prob_cpu.chunk_len.numpy(), prob_cpu.num_q_heads)
+    print(compare(out, lse, prob_cpu, rows, "MLA padded rows, pages of %d" % block_size))
