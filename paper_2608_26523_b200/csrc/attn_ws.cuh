@@ -288,12 +288,12 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                         const uint32_t ph = (kv_it / kWsStages) & 1;
                         const uint32_t dst = sKV + st * kTileBytes;
                         const uint32_t full = bar_kv_full + 8 * st;
+                        const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+                        const CUtensorMap* tm2 = which == 0 ? &tm_k2 : &tm_v2;
                         if (lane == 0) {
                             ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
                             if (ok) {
                                 mbar_arrive_expect_tx(full, kTileBytes);
-                                const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-                                const CUtensorMap* tm2 = which == 0 ? &tm_k2 : &tm_v2;
                                 if (kv_box_rows == kTileN) {
                                     int blk, slot_in;
                                     if (p.block_table == nullptr) {
@@ -308,26 +308,34 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                                         slot_in = 0;
                                     }
                                     tma_load_5d(dst, tm2, full, 0, slot_in, 0, g, blk);
-                                } else
-                                for (int off = 0; off < kTileN; off += kv_box_rows) {
-                                    const int pos = tile0 + off;
-                                    int blk, slot_in;
-                                    if (p.block_table == nullptr) {
-                                        blk = u.req;
-                                        slot_in = pos;
-                                    } else if (pos < u.kv_len) {
-                                        blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
-                                                    (pos >> p.block_shift));
-                                        slot_in = pos & ((1 << p.block_shift) - 1);
-                                    } else {
-                                        blk = p.num_blocks;  // out of range: the copy engine fills zeros
-                                        slot_in = 0;
-                                    }
-                                    const uint32_t o = static_cast<uint32_t>(off) * 128u;
-                                    tma_load_4d(dst + o, tm, full, 0, slot_in, g, blk);
-                                    tma_load_4d(dst + kSlabBytes + o, tm, full, 64, slot_in, g, blk);
                                 }
                             }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) break;
+                        if (kv_box_rows != kTileN) {
+                            // Pages smaller than a KV tile: one copy per (page, 64-column slab), each issued by a lane of its
+                            // own -- every lane looks up its page itself, and a lane's copy costs the warp a third of what a
+                            // single thread spends on one with its address arithmetic.  (The byte count was posted above.)
+                            const int per = kTileN / kv_box_rows;             // pages per tile: 2 .. 8
+                            if (lane < 2 * per) {
+                                const int off = (lane >> 1) * kv_box_rows, sl = lane & 1;
+                                const int pos = tile0 + off;
+                                int blk, slot_in;
+                                if (p.block_table == nullptr) {
+                                    blk = u.req;
+                                    slot_in = pos;
+                                } else if (pos < u.kv_len) {
+                                    blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                                (pos >> p.block_shift));
+                                    slot_in = pos & ((1 << p.block_shift) - 1);
+                                } else {
+                                    blk = p.num_blocks;  // out of range: the copy engine fills zeros
+                                    slot_in = 0;
+                                }
+                                tma_load_4d(dst + sl * kSlabBytes + static_cast<uint32_t>(off) * 128u, tm, full, sl * 64, slot_in, g, blk);
+                            }
+                            __syncwarp();
                         }
                         ok = __shfl_sync(0xffffffffu, ok, 0);
                         if (!ok) break;
