@@ -173,7 +173,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_item_full + 8 * i, 1);
-            mbar_init(bar_item_empty + 8 * i, 9);
+            mbar_init(bar_item_empty + 8 * i, kv_box_rows <= 32 ? 10 : 9);   // 8 softmax warps, the MMA thread, (the second producer)
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_p_full + 8 * i, 4);   // one arrival per softmax warp
             for (int c = 0; c < 3; ++c) mbar_init(bar_p_part + 16 * c + 8 * i, 4);
@@ -223,6 +223,92 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kWsRegsLow));
+        // One K (which = 0) or V (which = 1) tile of the item into the next ring stage, by the calling warp.
+        auto load_kv_tile = [&](const WorkUnit& u, int g, int tile0, int which, uint32_t kv_it, uint32_t& vfix_cnt) -> bool {
+            bool ok = true;
+                const uint32_t st = kv_it % kWsStages;
+                const uint32_t ph = (kv_it / kWsStages) & 1;
+                const uint32_t dst = sKV + st * kTileBytes;
+                const uint32_t full = bar_kv_full + 8 * st;
+                const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
+                const CUtensorMap* tm2 = which == 0 ? &tm_k2 : &tm_v2;
+                if (lane == 0) {
+                    ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
+                    if (ok) {
+                        mbar_arrive_expect_tx(full, kTileBytes);
+                        if (kv_box_rows == kTileN) {
+                            int blk, slot_in;
+                            if (p.block_table == nullptr) {
+                                blk = u.req;
+                                slot_in = tile0;
+                            } else if (tile0 < u.kv_len) {
+                                blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                            (tile0 >> p.block_shift));
+                                slot_in = tile0 & ((1 << p.block_shift) - 1);
+                            } else {
+                                blk = p.num_blocks;
+                                slot_in = 0;
+                            }
+                            tma_load_5d(dst, tm2, full, 0, slot_in, 0, g, blk);
+                        }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) return false;
+                if (kv_box_rows != kTileN) {
+                    // Pages smaller than a KV tile: one copy per (page, 64-column slab), each issued by a lane of its
+                    // own -- every lane looks up its page itself, and a lane's copy costs the warp a third of what a
+                    // single thread spends on one with its address arithmetic.  (The byte count was posted above.)
+                    const int per = kTileN / kv_box_rows;             // pages per tile: 2 .. 8
+                    if (lane < 2 * per) {
+                        const int off = (lane >> 1) * kv_box_rows, sl = lane & 1;
+                        const int pos = tile0 + off;
+                        int blk, slot_in;
+                        if (p.block_table == nullptr) {
+                            blk = u.req;
+                            slot_in = pos;
+                        } else if (pos < u.kv_len) {
+                            blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                        (pos >> p.block_shift));
+                            slot_in = pos & ((1 << p.block_shift) - 1);
+                        } else {
+                            blk = p.num_blocks;  // out of range: the copy engine fills zeros
+                            slot_in = 0;
+                        }
+                        tma_load_4d(dst + sl * kSlabBytes + static_cast<uint32_t>(off) * 128u, tm, full, sl * 64, slot_in, g, blk);
+                    }
+                    __syncwarp();
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) return false;
+                if (which == 1 && tile0 + kTileN > u.kv_len) {
+                    // Keys at or beyond kv_len do not exist; zero their V rows so that 0 * garbage
+                    // cannot poison O.  The MMA warp waits for bar_vfix on such a tile.
+                    if (lane == 0) ok = mbar_wait(full, ph, s_abort, 204);
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) return false;
+                    uint8_t* vb = gen_base + 2 * kTileBytes + st * kTileBytes;
+                    const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
+                    const uint4 z = make_uint4(0, 0, 0, 0);
+                    for (int r = first + lane; r < kTileN; r += 32) {
+                        uint4* a = reinterpret_cast<uint4*>(vb + r * 128);
+                        uint4* b = reinterpret_cast<uint4*>(vb + kSlabBytes + r * 128);
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            a[c] = z;
+                            b[c] = z;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_vfix + 24 * (vfix_cnt & 1));
+                    ++vfix_cnt;
+                }
+            return true;
+        };
+        // With pages of at most 32 tokens a tile takes 8 to 16 copies, and one warp issuing those of K and of V does not
+        // keep up: warp 2 then loads the V tiles (and zeroes their tails), warp 0 the K tiles.
+        const bool split_v = kv_box_rows <= 32;
         if (warp == 0) {
             // ============================ scheduler + TMA producer ============================
             uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_cnt = 0;
@@ -281,89 +367,36 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 ++q_it;
 
                 for (int j = u.kv_begin; j < u.kv_end && ok; ++j) {
-                    const int tile0 = j * kTileN;
 #pragma unroll
                     for (int which = 0; which < 2; ++which) {  // 0: K, 1: V
-                        const uint32_t st = kv_it % kWsStages;
-                        const uint32_t ph = (kv_it / kWsStages) & 1;
-                        const uint32_t dst = sKV + st * kTileBytes;
-                        const uint32_t full = bar_kv_full + 8 * st;
-                        const CUtensorMap* tm = which == 0 ? &tm_k : &tm_v;
-                        const CUtensorMap* tm2 = which == 0 ? &tm_k2 : &tm_v2;
-                        if (lane == 0) {
-                            ok = mbar_wait(bar_kv_empty + 8 * st, ph ^ 1, s_abort, 203);
-                            if (ok) {
-                                mbar_arrive_expect_tx(full, kTileBytes);
-                                if (kv_box_rows == kTileN) {
-                                    int blk, slot_in;
-                                    if (p.block_table == nullptr) {
-                                        blk = u.req;
-                                        slot_in = tile0;
-                                    } else if (tile0 < u.kv_len) {
-                                        blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
-                                                    (tile0 >> p.block_shift));
-                                        slot_in = tile0 & ((1 << p.block_shift) - 1);
-                                    } else {
-                                        blk = p.num_blocks;
-                                        slot_in = 0;
-                                    }
-                                    tma_load_5d(dst, tm2, full, 0, slot_in, 0, g, blk);
-                                }
-                            }
-                        }
-                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!(split_v && which == 1)) ok = load_kv_tile(u, g, j * kTileN, which, kv_it, vfix_cnt);
                         if (!ok) break;
-                        if (kv_box_rows != kTileN) {
-                            // Pages smaller than a KV tile: one copy per (page, 64-column slab), each issued by a lane of its
-                            // own -- every lane looks up its page itself, and a lane's copy costs the warp a third of what a
-                            // single thread spends on one with its address arithmetic.  (The byte count was posted above.)
-                            const int per = kTileN / kv_box_rows;             // pages per tile: 2 .. 8
-                            if (lane < 2 * per) {
-                                const int off = (lane >> 1) * kv_box_rows, sl = lane & 1;
-                                const int pos = tile0 + off;
-                                int blk, slot_in;
-                                if (p.block_table == nullptr) {
-                                    blk = u.req;
-                                    slot_in = pos;
-                                } else if (pos < u.kv_len) {
-                                    blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
-                                                (pos >> p.block_shift));
-                                    slot_in = pos & ((1 << p.block_shift) - 1);
-                                } else {
-                                    blk = p.num_blocks;  // out of range: the copy engine fills zeros
-                                    slot_in = 0;
-                                }
-                                tma_load_4d(dst + sl * kSlabBytes + static_cast<uint32_t>(off) * 128u, tm, full, sl * 64, slot_in, g, blk);
-                            }
-                            __syncwarp();
-                        }
-                        ok = __shfl_sync(0xffffffffu, ok, 0);
-                        if (!ok) break;
-                        if (which == 1 && tile0 + kTileN > u.kv_len) {
-                            // Keys at or beyond kv_len do not exist; zero their V rows so that 0 * garbage
-                            // cannot poison O.  The MMA warp waits for bar_vfix on such a tile.
-                            if (lane == 0) ok = mbar_wait(full, ph, s_abort, 204);
-                            ok = __shfl_sync(0xffffffffu, ok, 0);
-                            if (!ok) break;
-                            uint8_t* vb = gen_base + 2 * kTileBytes + st * kTileBytes;
-                            const int first = u.kv_len > tile0 ? u.kv_len - tile0 : 0;
-                            const uint4 z = make_uint4(0, 0, 0, 0);
-                            for (int r = first + lane; r < kTileN; r += 32) {
-                                uint4* a = reinterpret_cast<uint4*>(vb + r * 128);
-                                uint4* b = reinterpret_cast<uint4*>(vb + kSlabBytes + r * 128);
-#pragma unroll
-                                for (int c = 0; c < 8; ++c) {
-                                    a[c] = z;
-                                    b[c] = z;
-                                }
-                            }
-                            fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(bar_vfix + 24 * (vfix_cnt & 1));
-                            ++vfix_cnt;
-                        }
                         ++kv_it;
                     }
+                }
+                if (!ok) break;
+            }
+        } else if (warp == 2 && split_v) {
+            // ============================ second producer: the V tiles when pages are small ============================
+            // (follows the item ring like every other role)
+            uint32_t item_it = 0, kv_it = 0, vfix_cnt = 0;
+            while (true) {
+                const uint32_t slot = item_it & 1;
+                bool ok = true;
+                if (lane == 0) ok = mbar_wait(bar_item_full + 8 * slot, (item_it >> 1) & 1, s_abort, 211);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                const WorkUnit u = ring[slot].u;
+                const int g = ring[slot].h0 / G;
+                const int valid = ring[slot].valid;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_item_empty + 8 * slot);
+                ++item_it;
+                if (!valid) break;
+                for (int j = u.kv_begin; j < u.kv_end && ok; ++j) {
+                    ++kv_it;                                             // (the K tile: warp 0's)
+                    ok = load_kv_tile(u, g, j * kTileN, 1, kv_it, vfix_cnt);
+                    ++kv_it;
                 }
                 if (!ok) break;
             }
