@@ -338,6 +338,48 @@ def bench_groups(args):
     return 0
 
 
+def bench_pages(args):
+    """Cache page sizes: the cfg 2 chunk (8192 rows at prefix 32768) over caches of 256- to 16-token pages, and the cfg 3 chunk
+    (absorbed MLA) over 64- to 16-token pages.  A KV tile of 128 keys takes one copy per operand with pages of 128 tokens or
+    more and 2 x 128 / B copies with smaller ones."""
+    from paper_2608_26523_b200 import api
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    peaks = load_peaks()
+    prefix, chunk = (int(args.prefixes.split(",")[0]) if args.prefixes else 32768), 8192
+    stream = torch.cuda.Stream()
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    launches = 0
+    cases = [("d=128 (Hq=64 Hkv=4)", bs, (W.BASE_SEED + 2, 64, 4, 128, 128, 1.0, None, False)) for bs in (256, 128, 64, 32, 16)]
+    cases += [("absorbed MLA (Hq=128, 576/512)", bs, (W.BASE_SEED + 3, 128, 1, 576, 512, 0.5, 1.0 / math.sqrt(192.0), True))
+              for bs in (64, 32, 16)]
+    for desc, bs, (seed, hq, hkv, dqk, dv, std, scale, alias) in cases:
+        prob = W.single_request_cache(seed, prefix, chunk, hq, hkv, dqk, dv, bs, std, scale, alias, dev, "pages", prefix)
+        runner = api.ChunkAttn(prob, num_kv_splits=args.splits)
+        per, step_ms, nl, _ = time_points([runner], stream, max(args.steps, 5), max(args.warmup, 3))
+        launches += nl * max(args.steps, 5)
+        tf = prob.flops() / (per[0] * 1e-3) / 1e12
+        rows.append({"case": "%s, pages of %d tokens" % (desc, bs), "ms": round(per[0], 4), "tflops": round(tf, 1),
+                     "frac_of_burst": round(tf / peaks["bf16_tflops"], 4)})
+        del prob, runner
+        torch.cuda.empty_cache()
+    clocks = sampler.stop()
+    top = rows[1]
+    print(json.dumps({"metric": "chunk attention TFLOP/s by cache page size (1 B200)", "value": top["tflops"], "unit": UNIT, "n_gpus": 1,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": top["ms"], "higher_is_better": True, "dtype": "bf16",
+                      "data": "synthetic", "vs_baseline": None,
+                      "config": {"workload": "pages; chunk %d at prefix %d; %s" % (chunk, prefix, top["case"]),
+                                 "l2": "K/V of the d=128 cases is 84 MB, Q and out 134 MB each: larger than the L2 together"},
+                      "cases": rows,
+                      "roofline": {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": UNIT,
+                                   "frac": top["frac_of_burst"], "traffic": None,
+                                   "peak_source": "%s (burst bf16 matmul)" % peaks["_source"], "kernel": "attn128_ws_kernel, " + top["case"]},
+                      "gpu_launches": launches, "clocks": clocks}))
+    return 0
+
+
 def bench_merge(args):
     """vpp_lse_merge against the HBM roofline: S*(4*Dv+4) bytes read + (2*Dv+4) written per (row, head), CUDA-event timed,
     cycling through enough distinct buffers that no launch finds its inputs in the L2."""
@@ -617,7 +659,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse", "merge", "groups"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "append", "decode", "sparse", "merge", "groups", "pages"],
                     help="cfg2 is the benchmark the metric is quoted on; the others are the parity configurations")
     ap.add_argument("--prefixes", default="")
     ap.add_argument("--splits", type=int, default=0)
@@ -639,6 +681,8 @@ def main():
         return bench_sparse(args)
     if args.workload == "merge":
         return bench_merge(args)
+    if args.workload == "pages":
+        return bench_pages(args)
     if args.workload == "groups":
         return bench_groups(args)
     WL = {"cfg1": dict(prefixes=[0, 512, 1024, 1536], chunk=512, hq=4, hkv=1,

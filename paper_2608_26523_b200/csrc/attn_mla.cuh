@@ -172,53 +172,80 @@ attn_mla_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int pass = 0; pass < 2 && ok; ++pass) {
                 for (int j = t_lo; j < t_hi && ok; ++j) {
                     const int tile0 = j * kMlaTileN;
-                    if (lane == 0) {
-                        // page lookup once per tile (not per slab): a dependent global load costs more than a slab's MMAs
-                        int blk[4], slot_in[4];
-                        int np = 0;
-                        for (int off = 0; off < kMlaTileN; off += kv_box_rows, ++np) {
-                            const int pos = tile0 + off;
+                    if (kv_box_rows == kMlaTileN) {
+                        if (lane == 0) {
+                            // page lookup once per tile (not per slab): a dependent global load costs more than a slab's MMAs
+                            int blk, slot_in;
                             if (p.block_table == nullptr) {
-                                blk[np] = u.req;
-                                slot_in[np] = pos;
-                            } else if (pos < u.kv_len) {
-                                blk[np] = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
-                                                (pos >> p.block_shift));
-                                slot_in[np] = pos & ((1 << p.block_shift) - 1);
+                                blk = u.req;
+                                slot_in = tile0;
+                            } else if (tile0 < u.kv_len) {
+                                blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req +
+                                            (tile0 >> p.block_shift));
+                                slot_in = tile0 & ((1 << p.block_shift) - 1);
                             } else {
-                                blk[np] = p.num_blocks;  // out of range: the copy engine fills zeros
-                                slot_in[np] = 0;
+                                blk = p.num_blocks;  // out of range: the copy engine fills zeros
+                                slot_in = 0;
                             }
-                        }
-                        if (j == t_lo) {
-                            // the physical slabs change groups between passes: both groups of the previous tile
-                            // must have been released before anything of this pass is loaded
-                            ok = mbar_wait(bar_k_empty + 8, (fill & 1) ^ 1, s_abort, 505);
-                        }
-                        for (int grp = 0; grp < 2 && ok; ++grp) {
-                            ok = mbar_wait(bar_k_empty + 8 * grp, (fill & 1) ^ 1, s_abort, 503);
-                            if (!ok) break;
-                            const uint32_t full = bar_k_full + 8 * grp;
-                            const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
-                            mbar_arrive_expect_tx(full, (i1 - i0) * kMlaKSlab);
-                            if (kv_box_rows == kMlaTileN) {
+                            if (j == t_lo) {
+                                // the physical slabs change groups between passes: both groups of the previous tile
+                                // must have been released before anything of this pass is loaded
+                                ok = mbar_wait(bar_k_empty + 8, (fill & 1) ^ 1, s_abort, 505);
+                            }
+                            for (int grp = 0; grp < 2 && ok; ++grp) {
+                                ok = mbar_wait(bar_k_empty + 8 * grp, (fill & 1) ^ 1, s_abort, 503);
+                                if (!ok) break;
+                                const uint32_t full = bar_k_full + 8 * grp;
+                                const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
+                                mbar_arrive_expect_tx(full, (i1 - i0) * kMlaKSlab);
                                 // one page per tile: whole runs of consecutive slabs per instruction
                                 if (grp == 1) {
-                                    tma_load_5d(sK + pass * 4 * kMlaKSlab, &tm_k4, full, 0, slot_in[0], pass * 4, 0, blk[0]);
+                                    tma_load_5d(sK + pass * 4 * kMlaKSlab, &tm_k4, full, 0, slot_in, pass * 4, 0, blk);
                                 } else if (pass == 0) {
-                                    tma_load_5d(sK + 4 * kMlaKSlab, &tm_k5, full, 0, slot_in[0], 4, 0, blk[0]);
+                                    tma_load_5d(sK + 4 * kMlaKSlab, &tm_k5, full, 0, slot_in, 4, 0, blk);
                                 } else {
-                                    tma_load_5d(sK, &tm_k4, full, 0, slot_in[0], 0, 0, blk[0]);
-                                    tma_load_4d(sK + 8 * kMlaKSlab, &tm_k, full, 64 * 8, slot_in[0], 0, blk[0]);
-                                }
-                            } else {
-                                for (int i = i0; i < i1; ++i) {
-                                    const int s = mla_slab_order(pass, i);
-                                    for (int q = 0; q < np; ++q)
-                                        tma_load_4d(sK + s * kMlaKSlab + q * kv_box_rows * 128, &tm_k, full, 64 * s,
-                                                    slot_in[q], 0, blk[q]);
+                                    tma_load_5d(sK, &tm_k4, full, 0, slot_in, 0, 0, blk);
+                                    tma_load_4d(sK + 8 * kMlaKSlab, &tm_k, full, 64 * 8, slot_in, 0, blk);
                                 }
                             }
+                        }
+                    } else {
+                        // Pages smaller than the tile: one copy per (slab, page), each issued by a lane of its own (every lane
+                        // looks up the page of its copy itself) -- a single thread issuing the 18 to 36 copies of a tile one
+                        // after the other is several times slower than the MMAs that consume them.
+                        const int np = kMlaTileN / kv_box_rows;          // pages per tile: 2 or 4
+                        const int pq = lane % np;                          // this lane's page of the tile
+                        const int pos = tile0 + pq * kv_box_rows;
+                        int blk, slot_in;
+                        if (p.block_table == nullptr) {
+                            blk = u.req;
+                            slot_in = pos;
+                        } else if (pos < u.kv_len) {
+                            blk = __ldg(p.block_table + static_cast<long long>(u.req) * p.max_blocks_per_req + (pos >> p.block_shift));
+                            slot_in = pos & ((1 << p.block_shift) - 1);
+                        } else {
+                            blk = p.num_blocks;  // out of range: the copy engine fills zeros
+                            slot_in = 0;
+                        }
+                        if (j == t_lo) {
+                            if (lane == 0) ok = mbar_wait(bar_k_empty + 8, (fill & 1) ^ 1, s_abort, 505);
+                            ok = __shfl_sync(0xffffffffu, ok, 0);
+                        }
+                        for (int grp = 0; grp < 2 && ok; ++grp) {
+                            const uint32_t full = bar_k_full + 8 * grp;
+                            const int i0 = grp == 0 ? 0 : 5, i1 = grp == 0 ? 5 : 9;
+                            if (lane == 0) {
+                                ok = mbar_wait(bar_k_empty + 8 * grp, (fill & 1) ^ 1, s_abort, 503);
+                                if (ok) mbar_arrive_expect_tx(full, (i1 - i0) * kMlaKSlab);
+                            }
+                            ok = __shfl_sync(0xffffffffu, ok, 0);
+                            if (!ok) break;
+                            const int i = i0 + lane / np;
+                            if (i < i1) {
+                                const int sl = mla_slab_order(pass, i);
+                                tma_load_4d(sK + sl * kMlaKSlab + pq * kv_box_rows * 128, &tm_k, full, 64 * sl, slot_in, 0, blk);
+                            }
+                            __syncwarp();
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);

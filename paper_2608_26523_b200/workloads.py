@@ -215,6 +215,9 @@ def _single_request_cache(seed, max_prefix, chunk, hq, hkv, dqk, dv, block_size,
     return prob
 
 
+single_request_cache = _single_request_cache   # (same recipe with other shapes / page sizes: bench.py --workload pages)
+
+
 def cfg2(prefix=65536, max_prefix=None, device="cpu"):
     """GQA long-context chunk: Hq=64, Hkv=4, d=128, chunk 8192, 128-token pages, shuffled table."""
     mp = prefix if max_prefix is None else max_prefix
