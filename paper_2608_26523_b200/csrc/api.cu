@@ -310,10 +310,11 @@ int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
 // The d = 128 kernel pairs two q-heads of one kv-head per work item; when a kv-head's group is odd (MHA included) an
 // item is two consecutive 128-row query tiles of one q-head instead (work units of 256 rows).
 bool pairs_two_heads(const vpp_chunk_attn_args* a) { return (a->num_q_heads / a->num_kv_heads) % 2 == 0; }
-// The pair-of-SMs MLA kernel needs every 64-key group of a KV tile inside one page; smaller pages take the
+// The pair-of-SMs MLA kernel takes pages of 16 tokens and more (a 64-key group of a KV tile is one copy per slab group
+// with pages of 64 tokens or more, one copy per slab and page with smaller ones); still smaller pages take the
 // single-CTA two-pass kernel.
 bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
-    return (a->block_table == nullptr || a->block_size >= 64) && sm_count_or_default() >= 2;
+    return (a->block_table == nullptr || a->block_size >= 16) && sm_count_or_default() >= 2;
 }
 int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     if (fam == Family::kMla576) return 1;
@@ -517,8 +518,10 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
                                static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
         const uint64_t sk[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
                                 static_cast<uint64_t>(a->k_block_stride) * 2};
-        const uint32_t b3[5] = {vpp::kMla2BoxCols, vpp::kMla2BoxRows, vpp::kKG, 1, 1};               // one K hand-back group
-        const uint32_t b2[5] = {vpp::kMla2BoxCols, vpp::kMla2BoxRows, vpp::kMla2VBoxSlabs, 1, 1};    // one V chunk
+        // (with pages under 64 tokens the kernel copies page by page through tm_k and these two maps go unused)
+        const uint32_t krows = static_cast<uint32_t>(paged && B < vpp::kMla2BoxRows ? B : vpp::kMla2BoxRows);
+        const uint32_t b3[5] = {vpp::kMla2BoxCols, krows, vpp::kKG, 1, 1};               // one K hand-back group
+        const uint32_t b2[5] = {vpp::kMla2BoxCols, krows, vpp::kMla2VBoxSlabs, 1, 1};    // one V chunk
         if (!make_tmap(&tm_q9, a->q, 4, dq, sq, bq) ||
             !make_tmap(&tm_k93, a->k_cache, 5, d, sk, b3) || !make_tmap(&tm_k92, a->k_cache, 5, d, sk, b2))
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla pair) failed");
@@ -605,7 +608,7 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
     if (mla_pair) {
         auto kern = vpp::attn_mla2_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
-        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_qh9, tm_k93, tm_k92, ap);
+        if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_qh9, tm_k93, tm_k92, tm_k, ap, box_rows);
     } else if (fam == Family::kMla576) {
         auto kern = vpp::attn_mla_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);

@@ -186,7 +186,10 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kMla2Threads, 1)
 attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constant__ CUtensorMap tm_qh,
-                 const __grid_constant__ CUtensorMap tm_k3, const __grid_constant__ CUtensorMap tm_k2, const AttnParams p) {
+                 const __grid_constant__ CUtensorMap tm_k3, const __grid_constant__ CUtensorMap tm_k2,
+                 const __grid_constant__ CUtensorMap tm_k1, const AttnParams p, const int kv_box_rows) {
+    // tm_k1: (64 cols, keys, head, block) box (64, kv_box_rows, 1, 1) -- one page's share of one slab, for pages under 64 tokens
+    //        (kv_box_rows < 64): a 64-key group then takes one copy per (slab, page), each issued by a lane of its own
     // tm_qh: (64 cols, Hq heads, 9 slabs, T rows) box (64, 64, 9, 1)      -- 64 q-heads of one token (packed items)
     // tm_q1: (64 cols, T rows, 9 slabs, Hq) box (64, 64, 9, 1)         -- 64 query rows, all nine 64-column slabs
     // tm_k3: (64 cols, keys, 9 slabs, head, block) box (64, 64, 3, 1, 1) -- 64 keys of three slabs: one K hand-back group
@@ -328,7 +331,52 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
     if (warp == 0) {
         // ===================================== Q / K producer =====================================
         // one thread: group g of the next tile is requested as soon as the MMAs that read group g of this tile are done
-        if (lane == 0) {
+        if (kv_box_rows < 64) {
+            // pages under 64 tokens: the waits and the Q copy by lane 0, the K copies of a group by 3 x (64 / page) lanes
+            const int np = 64 / kv_box_rows, pq = lane % np;
+            uint32_t q_it = 0, kc = 0;
+            bool ok = true;
+            for (int item = pair; item < total_items && ok; item += num_pairs) {
+                WorkUnit u;
+                int h;
+                if (!get_item(item, u, h)) continue;
+                if (lane == 0) {
+                    if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 801);
+                    if (ok) {
+                        if (leader) mbar_arrive_expect_tx(bar_q_full, 2 * kMla2QBytes);
+                        if (is_packed(u))
+                            tma2_load_4d(sQ, &tm_qh, pair_q_full, 0, static_cast<int>(rank) * kMla2Rows, 0, u.q_row0);
+                        else
+                            tma2_load_4d(sQ, &tm_q1, pair_q_full, 0, u.q_row0 + static_cast<int>(rank) * kMla2Rows, 0, h);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                ++q_it;
+                const int t_hi = tile_hi(u);
+                for (int j = u.kv_begin; j < t_hi && ok; ++j) {
+                    int blk, slot_in;                      // this lane's page of the CTA's 64 keys
+                    page_of(u, j * kTileN + static_cast<int>(rank) * 64 + pq * kv_box_rows, blk, slot_in);
+                    const uint32_t par = (kc & 1) ^ 1;
+#pragma unroll 1
+                    for (int g = 0; g < kKGroups; ++g) {
+                        if (lane == 0) {
+                            if (g < kKGroups - 1) ok = mbar_wait(bar_k_empty + 8 * g, par, s_abort, 802);
+                            else if (kc > 0) ok = mbar_wait(bar_s_full + 8 * ((kc - 1) & 1), ((kc - 1) >> 1) & 1, s_abort, 802);
+                            if (ok && leader) mbar_arrive_expect_tx(bar_k_full + 8 * g, 2 * kKG * 8192);
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) break;
+                        if (lane < kKG * np) {
+                            const int sl = g * kKG + lane / np;
+                            tma2_load_4d(sK + sl * 8192 + pq * kv_box_rows * 128, &tm_k1, pair_k_full + 8 * g, 64 * sl, slot_in, 0, blk);
+                        }
+                        __syncwarp();
+                    }
+                    ++kc;
+                }
+            }
+        } else if (lane == 0) {
             uint32_t q_it = 0, kc = 0, item_it = 0;
             bool ok = true;
             for (int item = pair; item < total_items && ok; item += num_pairs) {
@@ -387,7 +435,34 @@ attn_mla2_kernel(const __grid_constant__ CUtensorMap tm_q1, const __grid_constan
             for (int j = u.kv_begin; j < t_hi && ok; ++j) {
                 const int tile0 = j * kTileN;
                 const bool tail = tile0 + kTileN > u.kv_len;
-                if (lane == 0) {
+                if (kv_box_rows < 64) {
+                    // pages under 64 tokens: a group's two chunks take 2 chunks x 2 slabs x (64 / page) copies, a lane each
+                    const int np = 64 / kv_box_rows, pq = lane % np;
+                    const uint32_t par = (vc & 1) ^ 1;
+#pragma unroll 1
+                    for (int g = 0; g < kVGroups; ++g) {
+                        if (lane == 0) {
+                            if (g < kVGroups - 1) ok = mbar_wait(bar_v_empty + 8 * g, par, s_abort, 803);
+                            else if (vc > 0) ok = mbar_wait(bar_pv_done, (vc - 1) & 1, s_abort, 803);
+                            if (ok) {
+                                if (tail) mbar_arrive_expect_tx(own_v_full + 8 * g, kVG * kMla2VChunk);
+                                else if (leader) mbar_arrive_expect_tx(bar_v_full + 8 * g, 2 * kVG * kMla2VChunk);
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (!ok) break;
+                        if (lane < kVG * 2 * np) {
+                            const int c = g * kVG + lane / (2 * np), s2 = (lane / np) & 1;
+                            const int hf = c >> 1, slab = 4 * (c & 1) + 2 * static_cast<int>(rank) + s2;
+                            int blk, slot_in;
+                            page_of(u, tile0 + 64 * hf + pq * kv_box_rows, blk, slot_in);
+                            const uint32_t dst = sV + c * kMla2VChunk + s2 * 8192 + pq * kv_box_rows * 128;
+                            if (tail) tma_load_4d(dst, &tm_k1, own_v_full + 8 * g, 64 * slab, slot_in, 0, blk);
+                            else tma2_load_4d(dst, &tm_k1, pair_v_full + 8 * g, 64 * slab, slot_in, 0, blk);
+                        }
+                        __syncwarp();
+                    }
+                } else if (lane == 0) {
                     const int b0 = nb0, s0 = ns0, b1 = nb1, s1 = ns1;
                     if (j + 1 < t_hi) {
                         page_of(u, tile0 + kTileN, nb0, ns0);
