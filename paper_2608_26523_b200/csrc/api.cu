@@ -10,7 +10,6 @@
 #include <mutex>
 
 #include "../../include/vpp.h"
-#include "attn_mla.cuh"
 #include "attn_mla2.cuh"
 #include "attn_dsa.cuh"
 #include "attn_ws.cuh"
@@ -310,12 +309,8 @@ int choose_splits(const vpp_chunk_attn_args* a, int heads_per_item) {
 // The d = 128 kernel pairs two q-heads of one kv-head per work item; when a kv-head's group is odd (MHA included) an
 // item is two consecutive 128-row query tiles of one q-head instead (work units of 256 rows).
 bool pairs_two_heads(const vpp_chunk_attn_args* a) { return (a->num_q_heads / a->num_kv_heads) % 2 == 0; }
-// The pair-of-SMs MLA kernel takes pages of 16 tokens and more (a 64-key group of a KV tile is one copy per slab group
-// with pages of 64 tokens or more, one copy per slab and page with smaller ones); still smaller pages take the
-// single-CTA two-pass kernel.
-bool use_mla_pair_kernel(const vpp_chunk_attn_args* a) {
-    return (a->block_table == nullptr || a->block_size >= 16) && sm_count_or_default() >= 2;
-}
+// The absorbed-MLA kernel runs on pairs of SMs (2-CTA clusters).
+bool mla_kernel_available() { return sm_count_or_default() >= 2; }
 int heads_per_item(const vpp_chunk_attn_args* a, Family fam) {
     if (fam == Family::kMla576) return 1;
     return pairs_two_heads(a) ? 2 : 1;
@@ -445,12 +440,14 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
             return fail(VPP_ERR_CUDA, "memset status: %s", cudaGetErrorString(cudaGetLastError()));
     }
     if (a->total_q == 0 || a->num_reqs == 0) return VPP_OK;
+    if (fam == Family::kMla576 && !mla_kernel_available())
+        return fail(VPP_ERR_UNSUPPORTED, "the absorbed-MLA kernel needs clusters of two SMs");
 
     uint8_t* ws = static_cast<uint8_t*>(a->workspace);
     const bool paged = a->block_table != nullptr;
     const int B = paged ? a->block_size : a->max_seq_len;
     const int n_blocks = paged ? a->num_blocks : a->num_reqs;
-    const int tile_n = fam == Family::kMla576 ? vpp::kMlaTileN : vpp::kTileN;  // keys per KV tile of the kernel
+    const int tile_n = fam == Family::kMla576 ? vpp::kMla2BoxRows : vpp::kTileN;  // keys one copy can bring (MLA: a CTA's 64 of the pair's tile)
     const int box_rows = paged ? (B < tile_n ? B : tile_n) : tile_n;
 
     // ---- tensor maps ----
@@ -507,7 +504,7 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
             return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k/v tiles) failed");
     }
     CUtensorMap tm_q9, tm_qh9, tm_k93, tm_k92;  // 64 rows of one 64-column slab per box (tm_k93 / tm_k92: of 3 / 2 slabs)
-    const bool mla_pair = fam == Family::kMla576 && use_mla_pair_kernel(a);
+    const bool mla_pair = fam == Family::kMla576;
     if (mla_pair) {
         const uint64_t dq[4] = {64, static_cast<uint64_t>(a->total_q), static_cast<uint64_t>(vpp::kMlaSlabs),
                                 static_cast<uint64_t>(a->num_q_heads)};
@@ -533,20 +530,6 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
         const uint32_t bh[4] = {64, 64, static_cast<uint32_t>(vpp::kMlaSlabs), 1};   // heads past num_q_heads read as zero
         if (!make_tmap(&tm_qh9, a->q, 4, dh, sh, bh)) return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(mla q heads) failed");
     }
-    CUtensorMap tm_k4, tm_k5;
-    if (fam == Family::kMla576) {
-        // rank-5 views (64 columns, keys, slab, head, block): boxes of 4 / 5 slabs x 64 keys
-        const uint64_t d[5] = {64, static_cast<uint64_t>(B), static_cast<uint64_t>(vpp::kMlaSlabs),
-                               static_cast<uint64_t>(a->num_kv_heads), static_cast<uint64_t>(n_blocks)};
-        const uint64_t s[4] = {static_cast<uint64_t>(a->k_token_stride) * 2, 128, static_cast<uint64_t>(a->k_head_stride) * 2,
-                               static_cast<uint64_t>(a->k_block_stride) * 2};
-        const uint32_t rows = static_cast<uint32_t>(box_rows);
-        const uint32_t b4[5] = {64, rows, 4, 1, 1};
-        const uint32_t b5[5] = {64, rows, 5, 1, 1};
-        if (!make_tmap(&tm_k4, a->k_cache, 5, d, s, b4) || !make_tmap(&tm_k5, a->k_cache, 5, d, s, b5))
-            return fail(VPP_ERR_CUDA, "cuTensorMapEncodeTiled(k slab groups) failed");
-    }
-
     // ---- work decomposition ----
     int32_t* row_splits = reinterpret_cast<int32_t*>(ws + L.row_splits);
     vpp::PrepParams pp{};
@@ -609,10 +592,6 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
         auto kern = vpp::attn_mla2_kernel;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
         if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_qh9, tm_k93, tm_k92, tm_k, ap, box_rows);
-    } else if (fam == Family::kMla576) {
-        auto kern = vpp::attn_mla_kernel;
-        ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMlaSmemBytes);
-        if (ce == cudaSuccess) kern<<<sms, vpp::kMlaThreads, vpp::kMlaSmemBytes, stream>>>(tm_q, tm_k, tm_k4, tm_k5, ap, box_rows);
     } else {
         auto kern = pairs_two_heads(a) ? vpp::attn128_ws_kernel<false> : vpp::attn128_ws_kernel<true>;
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);

@@ -31,11 +31,13 @@
 #pragma once
 #include <type_traits>
 
-#include "attn_mla.cuh"  // kMla* constants
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace vpp {
+
+constexpr int kMlaDqk = 576, kMlaDv = 512;         // latent row: 512 value features + 64 rope features
+constexpr int kMlaSlabs = kMlaDqk / 64;            // 9 slabs of 64 features
 
 constexpr int kMla2Threads = 256;
 constexpr int kMla2Rows = 64;                                 // query rows per CTA
