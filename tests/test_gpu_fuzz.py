@@ -56,3 +56,24 @@ def test_random_batches(seed):
     out, lse, _ = run_gpu(prob.to("cuda"), c["splits"])
     rows = oracle.all_rows(prob.chunk_len.numpy(), prob.num_q_heads)
     print(c, compare(out, lse, prob, rows, "fuzz %d" % seed))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_batches_of_many_items(seed):
+    """Launches of several hundred to a few thousand work items (every CTA runs many, long and short ones in turn), d = 128
+    and MLA: item ring, K/V ring, tail fix-ups and barrier phases across item boundaries."""
+    rng = np.random.default_rng(7500 + seed)
+    mla = seed % 3 == 2
+    R = int(rng.integers(12, 48))
+    prefix = [int(rng.integers(0, 2500)) if rng.random() < 0.8 else 0 for _ in range(R)]
+    chunk = [1 if rng.random() < 0.3 else int(rng.integers(1, 330)) for _ in range(R)]
+    bs = int(rng.choice([16, 64, 128]))
+    if mla:
+        prob = W.make_problem(8500 + seed, prefix, chunk, 32, 1, 576, 512, block_size=bs, std=0.5, scale=1.0 / 192 ** 0.5,
+                              v_aliases_k=True)
+    else:
+        hkv = int(rng.choice([2, 4]))
+        prob = W.make_problem(8500 + seed, prefix, chunk, hkv * int(rng.choice([1, 4, 8])), hkv, 128, 128, block_size=bs, std=0.7)
+    out, lse, _ = run_gpu(prob.to("cuda"), int(rng.choice([0, 0, 2])))
+    rows = oracle.all_rows(prob.chunk_len.numpy(), prob.num_q_heads)
+    print(R, sum(chunk), bs, compare(out, lse, prob, rows, "fuzz many %d" % seed))
