@@ -593,7 +593,10 @@ vpp_status run_chunk_attn(const vpp_chunk_attn_args* a, vpp_stream_t stream_, co
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kMla2SmemBytes);
         if (ce == cudaSuccess) kern<<<(sms / 2) * 2, vpp::kMla2Threads, vpp::kMla2SmemBytes, stream>>>(tm_q9, tm_qh9, tm_k93, tm_k92, tm_k, ap, box_rows);
     } else {
-        auto kern = pairs_two_heads(a) ? vpp::attn128_ws_kernel<false> : vpp::attn128_ws_kernel<true>;
+        // a second producer warp for launches bound by the arrival of K/V: pages smaller than a KV tile, batches of decode rows
+        const bool v_warp = box_rows < vpp::kTileN || a->total_q <= a->num_reqs;
+        auto kern = pairs_two_heads(a) ? (v_warp ? vpp::attn128_ws_kernel<false, true> : vpp::attn128_ws_kernel<false, false>)
+                                       : (v_warp ? vpp::attn128_ws_kernel<true, true> : vpp::attn128_ws_kernel<true, false>);
         ce = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, vpp::kWsSmemBytes);
         if (ce == cudaSuccess) {
             // programmatic dependent launch: set-up overlaps the work-decomposition kernel (the kernel waits for it

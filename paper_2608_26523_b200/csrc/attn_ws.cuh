@@ -120,7 +120,7 @@ __device__ __noinline__ void ws_packed_merge(void* out, float* lse_out, float* o
     }
 }
 
-template <bool kSameHead>
+template <bool kSameHead, bool kVWarp>
 __global__ void __launch_bounds__(kWsThreads, 1)
 attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_q2,
@@ -173,7 +173,7 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (tid == 0) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar_item_full + 8 * i, 1);
-            mbar_init(bar_item_empty + 8 * i, kv_box_rows <= 32 ? 10 : 9);   // 8 softmax warps, the MMA thread, (the second producer)
+            mbar_init(bar_item_empty + 8 * i, kVWarp ? 10 : 9);   // 8 softmax warps, the MMA thread, (the second producer)
             mbar_init(bar_s_full + 8 * i, 1);
             mbar_init(bar_p_full + 8 * i, 4);   // one arrival per softmax warp
             for (int c = 0; c < 3; ++c) mbar_init(bar_p_part + 16 * c + 8 * i, 4);
@@ -306,9 +306,11 @@ attn128_ws_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 }
             return true;
         };
-        // With pages of at most 32 tokens a tile takes 8 to 16 copies, and one warp issuing those of K and of V does not
-        // keep up: warp 2 then loads the V tiles (and zeroes their tails), warp 0 the K tiles.
-        const bool split_v = kv_box_rows <= 32;
+        // kVWarp: a second producer warp (warp 2) loads the V tiles, warp 0 the K tiles.  The host chooses it for the launches
+        // that are bound by how fast K/V arrives: pages smaller than a KV tile (a tile is then 4 to 16 copies per operand)
+        // and batches of decode rows, which stream K/V at memory speed (+10 to 18 % with K and V requested by two warps).
+        // Prefill over large pages keeps the single producer (a second one costs it 1 to 2 %).
+        constexpr bool split_v = kVWarp;
         if (warp == 0) {
             // ============================ scheduler + TMA producer ============================
             uint32_t item_it = 0, q_it = 0, kv_it = 0, vfix_cnt = 0;
